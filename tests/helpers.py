@@ -1,0 +1,70 @@
+"""Test-side helpers: dtype plumbing and independent reference arithmetic."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import torch
+
+
+def bf16_bits(t):
+    """torch bf16 tensor -> numpy uint16 bit patterns (same shape)."""
+    assert t.dtype == torch.bfloat16
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def bits_to_f64(bits):
+    """numpy uint16 bf16 bit patterns -> float64 values."""
+    w = bits.astype(np.uint32) << 16
+    return w.view(np.float32).astype(np.float64)
+
+
+def frac_to_bf16(fr):
+    """Exact Fraction -> torch bf16 scalar; asserts it is representable."""
+    x = torch.tensor(float(fr), dtype=torch.float32).to(torch.bfloat16)
+    assert Fraction(float(x)) == Fraction(fr), f"{fr} is not exact in bf16"
+    return x
+
+
+def round_half_even(fr):
+    """Exact round-half-to-even of a Fraction."""
+    fl = math.floor(fr)
+    rem = fr - fl
+    if rem > Fraction(1, 2):
+        return fl + 1
+    if rem < Fraction(1, 2):
+        return fl
+    return fl if fl % 2 == 0 else fl + 1
+
+
+def exact_codes(row_f64):
+    """Exact rational quantiser of one row given as float64 values."""
+    fr = [Fraction(float(x)) for x in row_f64]
+    amax = max(abs(x) for x in fr)
+    if amax == 0:
+        return [0] * len(fr), Fraction(0)
+    codes = [max(-127, min(127, round_half_even(127 * x / amax))) for x in fr]
+    return codes, amax / 127
+
+
+def dense_attention(q, k_hat, v_hat, kv_len, sm_scale):
+    """Dense numpy fp64 softmax attention for one sequence.
+
+    q [nq, Hq, D], k_hat/v_hat [L, Hkv, D] float64 (already dequantised).
+    Builds the full masked score matrix per head and uses matrix products.
+    """
+    nq, Hq, D = q.shape
+    Hkv = k_hat.shape[1]
+    G = Hq // Hkv
+    out = np.zeros((nq, Hq, D))
+    jj = np.arange(kv_len)[None, :]
+    tt = np.arange(nq)[:, None]
+    visible = jj <= (kv_len - nq + tt)
+    for h in range(Hq):
+        g = h // G
+        S = sm_scale * (q[:, h, :] @ k_hat[:kv_len, g, :].T)
+        S = np.where(visible, S, -np.inf)
+        S = S - S.max(axis=1, keepdims=True)
+        P = np.exp(S)
+        P = P / P.sum(axis=1, keepdims=True)
+        out[:, h, :] = P @ v_hat[:kv_len, g, :]
+    return out
