@@ -1,0 +1,164 @@
+/*
+ * slim.h - C ABI of the SlimAttention / INT8 KV cache library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the attention hot path of "Inference Performance
+ * Optimization for Large Language Models on CPUs" (arXiv 2407.07304):
+ *   - Section 2.2: a KV cache stored as INT8 codes with one scale per token and
+ *     per head, consumed by a hybrid-dtype kernel that converts the codes on the
+ *     fly (there AVX-512 FMA; here tensor-core MMA);
+ *   - Section 2.1: SlimAttention, a one-dimensional decomposition of attention:
+ *     for a block of query rows the whole score row against all keys is formed,
+ *     softmaxed once, and multiplied by V.
+ * The paper does not fix the cache format; this library uses symmetric codes in
+ * [-127, 127], scale = absmax / 127 stored as fp32, round half to even.
+ *
+ * General rules
+ *   - Every pointer marked "device" must point to memory of the current CUDA
+ *     device; pointers marked "host" are ordinary host memory.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream).  Unless stated otherwise no call synchronises
+ *     with the host, allocates or frees memory, or keeps a pointer after it
+ *     returns.
+ *   - The caller owns every buffer.  The library never writes block_table or
+ *     any length array.
+ *   - Return value: SLIM_OK (0) or a negative SLIM_ERR_* code.  Arguments are
+ *     validated on the host before anything is launched; a call that returns an
+ *     error other than SLIM_ERR_CUDA has launched nothing.
+ *   - Supported shapes: head_dim == 128, page_tokens == 128, Hq % Hkv == 0 and
+ *     Hq / Hkv <= 16 for decode; Q and O are bf16.  Other shapes return
+ *     SLIM_ERR_UNSUPPORTED.
+ *   - Non-finite K/V/Q values are outside the contract.
+ */
+#ifndef SLIM_H_
+#define SLIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SLIM_OK               0
+#define SLIM_ERR_INVALID_ARG (-1)  /* null pointer, negative size, inconsistent sizes */
+#define SLIM_ERR_UNSUPPORTED (-2)  /* shape outside the supported set               */
+#define SLIM_ERR_WORKSPACE   (-3)  /* workspace missing or too small                */
+#define SLIM_ERR_CUDA        (-4)  /* a CUDA runtime call failed; see slim_last_cuda_error */
+#define SLIM_ERR_TIMEOUT     (-5)  /* a bounded device-side wait ran out            */
+
+#define SLIM_HEAD_DIM    128
+#define SLIM_PAGE_TOKENS 128
+
+#define SLIM_PHASE_PREFILL 0
+#define SLIM_PHASE_DECODE  1
+
+/*
+ * Paged INT8 KV cache of one attention layer (Section 2.2).  A page holds
+ * SLIM_PAGE_TOKENS consecutive token positions of one sequence, for every kv
+ * head.  Token position `pos` of sequence b lives in page
+ * block_table[b * max_pages_per_seq + pos / 128], slot pos % 128.
+ *
+ *   codes   device int8  [num_pages][num_kv_heads][2][128 slots][128 dims]   (index 0 = K, 1 = V)
+ *   scales  device fp32  [num_pages][num_kv_heads][2][128 slots]
+ *   block_table device int32 [B][max_pages_per_seq]; entries in [0, num_pages)
+ *
+ * A dequantised element is (float)code * scale of its (token, kv head).
+ * codes and scales must be 16-byte aligned.  The struct itself is host memory
+ * and is read during the call only.
+ */
+typedef struct slim_cache {
+    int8_t        *codes;
+    float         *scales;
+    const int32_t *block_table;
+    int32_t        num_pages;
+    int32_t        page_tokens;        /* must be 128 */
+    int32_t        num_kv_heads;
+    int32_t        head_dim;           /* must be 128 */
+    int32_t        max_pages_per_seq;
+} slim_cache_t;
+
+/*
+ * Quantise new K and V rows and write them into the cache (Section 2.2: INT8
+ * codes, "a unique scale for each token and each head").
+ *
+ * For each row x (128 bf16 values of one token and one kv head, K and V
+ * separately): amax = max|x_d|; scale = amax / 127 (fp32, correctly rounded);
+ * code_d = clamp(round_half_even(127 * x_d / amax), -127, 127); an all-zero row
+ * gets scale 0 and codes 0.  Codes and scale bits are reproducible exactly.
+ *
+ *   k_new, v_new  device bf16 [total_new][num_kv_heads][128], the new tokens of
+ *                 all sequences concatenated in sequence order; 8-byte aligned
+ *   cu_new        device int32 [B+1]: rows cu_new[b] .. cu_new[b+1]-1 belong to
+ *                 sequence b (cu_new[0] == 0)
+ *   start_pos     device int32 [B]: cache position of sequence b's first new token
+ *   B             number of sequences (>= 0; 0 is a no-op)
+ *   max_new       upper bound on cu_new[b+1]-cu_new[b] (sizes the launch)
+ *
+ * The pages addressed through block_table must exist; a position past
+ * max_pages_per_seq * 128 or a page id outside [0, num_pages) is skipped.
+ */
+int slim_kv_append(const slim_cache_t *cache, const void *k_new, const void *v_new,
+                   const int32_t *cu_new, const int32_t *start_pos,
+                   int32_t B, int32_t max_new, void *stream);
+
+/*
+ * Causal prefill attention over the INT8 cache (Section 2.1).  The new tokens'
+ * K/V must already be in the cache (slim_kv_append first).
+ *
+ * For sequence b with q_len = cu_q[b+1]-cu_q[b] query rows and kv_len[b] cached
+ * tokens, query row t (0-based) sees keys j <= kv_len[b] - q_len + t; query
+ * head h reads kv head h / (Hq / Hkv).  For each (row, head):
+ *   s_j = sm_scale * sum_d q_d * (k_code[j][d] * k_scale[j]);  p = softmax_j(s);
+ *   o_d = sum_j p_j * (v_code[j][d] * v_scale[j]).
+ * A row that sees no key gets zeros.
+ *
+ *   q      device bf16 [total_q][Hq][128], 16-byte aligned
+ *   out    device bf16 [total_q][Hq][128], 16-byte aligned
+ *   cu_q   device int32 [B+1];   kv_len device int32 [B]
+ *   max_q, max_kv  upper bounds on q_len and kv_len (size the launch)
+ *   workspace      device scratch of at least
+ *                  slim_workspace_bytes(SLIM_PHASE_PREFILL, ...) bytes (may be
+ *                  NULL when that size is 0)
+ */
+int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out,
+                      const int32_t *cu_q, const int32_t *kv_len,
+                      int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq, float sm_scale,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Decode attention: one query token per sequence against all kv_len[b] cached
+ * tokens (the new token's K/V already appended).  Same arithmetic as above with
+ * q_len == 1.  The next-token phase is a matrix-vector product bound by memory
+ * bandwidth (Section 2.2, Eq. 1); the key range is split across thread blocks
+ * and the pieces are merged by the log-sum-exp identity in a second kernel.
+ * A sequence with kv_len[b] == 0 gets zeros.
+ *
+ *   q, out   device bf16 [B][Hq][128], 16-byte aligned
+ *   kv_len   device int32 [B];  max_kv upper bound on kv_len (sizes the launch)
+ *   workspace device scratch of at least
+ *             slim_workspace_bytes(SLIM_PHASE_DECODE, ...) bytes, 16-byte
+ *             aligned; contents need not be initialised
+ */
+int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out,
+                     const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* Scratch bytes needed by a phase (SLIM_PHASE_*) for the given shape; 0 on invalid arguments. */
+size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q, int32_t max_kv);
+
+/* Bytes of the codes and scales arrays of a pool of num_pages pages
+ * (Eq. 1 with s_d = 1 for the codes, plus 2 fp32 scales per token and head). */
+size_t slim_cache_code_bytes(int32_t num_pages, int32_t num_kv_heads);
+size_t slim_cache_scale_bytes(int32_t num_pages, int32_t num_kv_heads);
+
+/* Text for a return code; never NULL. */
+const char *slim_strerror(int code);
+/* The cudaError_t value behind the calling thread's last SLIM_ERR_CUDA (0 if none). */
+int slim_last_cuda_error(void);
+/* Library version, major * 10000 + minor * 100 + patch. */
+int slim_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLIM_H_ */

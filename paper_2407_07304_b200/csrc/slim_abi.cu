@@ -1,0 +1,124 @@
+// C ABI of the library (declared in include/slim.h): argument validation and dispatch.
+#include "slim_common.cuh"
+
+#define SLIM_EXPORT extern "C" __attribute__((visibility("default")))
+
+namespace slim {
+
+static thread_local int g_last_cuda_error = 0;
+
+int set_cuda_error(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    return SLIM_ERR_CUDA;
+}
+
+int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
+                  const int32_t *start_pos, int B, int max_new, cudaStream_t stream);
+int launch_decode(const slim_cache_t *c, const void *q, void *out, const int32_t *kv_len, int B, int max_kv,
+                  int Hq, float sm_scale, void *workspace, cudaStream_t stream);
+size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
+int launch_prefill_mma(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
+                       int B, int max_q, int Hq, float sm_scale, cudaStream_t stream);
+
+static int check_cache(const slim_cache_t *c)
+{
+    if (c == nullptr || c->codes == nullptr || c->scales == nullptr || c->block_table == nullptr)
+        return SLIM_ERR_INVALID_ARG;
+    if (c->num_pages <= 0 || c->num_kv_heads <= 0 || c->max_pages_per_seq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (c->page_tokens != SLIM_PAGE_TOKENS || c->head_dim != SLIM_HEAD_DIM) return SLIM_ERR_UNSUPPORTED;
+    if (((uintptr_t)c->codes & 15) || ((uintptr_t)c->scales & 15)) return SLIM_ERR_INVALID_ARG;
+    return SLIM_OK;
+}
+
+}  // namespace slim
+
+using namespace slim;
+
+SLIM_EXPORT int slim_kv_append(const slim_cache_t *cache, const void *k_new, const void *v_new,
+                               const int32_t *cu_new, const int32_t *start_pos, int32_t B, int32_t max_new,
+                               void *stream)
+{
+    int rc = check_cache(cache);
+    if (rc != SLIM_OK) return rc;
+    if (B < 0 || max_new < 0) return SLIM_ERR_INVALID_ARG;
+    if (B == 0 || max_new == 0) return SLIM_OK;
+    if (k_new == nullptr || v_new == nullptr || cu_new == nullptr || start_pos == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)k_new & 7) || ((uintptr_t)v_new & 7)) return SLIM_ERR_INVALID_ARG;
+    if (B > 65535) return SLIM_ERR_UNSUPPORTED;
+    return launch_append(cache, k_new, v_new, cu_new, start_pos, B, max_new, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
+                                  const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
+                                  float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_cache(cache);
+    if (rc != SLIM_OK) return rc;
+    if (B < 0 || max_q < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (Hq % cache->num_kv_heads != 0) return SLIM_ERR_UNSUPPORTED;
+    if (B == 0 || max_q == 0) return SLIM_OK;
+    if (q == nullptr || out == nullptr || cu_q == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
+    if (B > 65535 || Hq > 65535) return SLIM_ERR_UNSUPPORTED;
+    if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
+    const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
+    if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
+    return launch_prefill_mma(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out, const int32_t *kv_len,
+                                 int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
+                                 size_t workspace_bytes, void *stream)
+{
+    int rc = check_cache(cache);
+    if (rc != SLIM_OK) return rc;
+    if (B < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (Hq % cache->num_kv_heads != 0 || Hq / cache->num_kv_heads > 16) return SLIM_ERR_UNSUPPORTED;
+    if (B == 0) return SLIM_OK;
+    if (q == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
+    if (B > 65535 || cache->num_kv_heads > 65535) return SLIM_ERR_UNSUPPORTED;
+    if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
+    const size_t need = slim_workspace_bytes(SLIM_PHASE_DECODE, B, Hq, cache->num_kv_heads, 1, max_kv);
+    if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 15) return SLIM_ERR_INVALID_ARG;
+    return launch_decode(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q,
+                                        int32_t max_kv)
+{
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || max_kv < 0 || max_q < 0) return 0;
+    if (phase == SLIM_PHASE_DECODE) return decode_workspace_bytes(B, Hq, Hkv, max_kv);
+    return 0;
+}
+
+SLIM_EXPORT size_t slim_cache_code_bytes(int32_t num_pages, int32_t num_kv_heads)
+{
+    if (num_pages <= 0 || num_kv_heads <= 0) return 0;
+    return (size_t)num_pages * num_kv_heads * 2 * SLIM_PAGE_TOKENS * SLIM_HEAD_DIM;
+}
+
+SLIM_EXPORT size_t slim_cache_scale_bytes(int32_t num_pages, int32_t num_kv_heads)
+{
+    if (num_pages <= 0 || num_kv_heads <= 0) return 0;
+    return (size_t)num_pages * num_kv_heads * 2 * SLIM_PAGE_TOKENS * sizeof(float);
+}
+
+SLIM_EXPORT const char *slim_strerror(int code)
+{
+    switch (code) {
+        case SLIM_OK: return "ok";
+        case SLIM_ERR_INVALID_ARG: return "invalid argument";
+        case SLIM_ERR_UNSUPPORTED: return "unsupported shape";
+        case SLIM_ERR_WORKSPACE: return "workspace missing or too small";
+        case SLIM_ERR_CUDA: return "CUDA runtime error";
+        case SLIM_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+SLIM_EXPORT int slim_last_cuda_error(void) { return g_last_cuda_error; }
+
+SLIM_EXPORT int slim_version(void) { return 100; }
