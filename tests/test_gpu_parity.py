@@ -1,0 +1,204 @@
+"""CUDA path vs the CPU oracle, through the C ABI, on the five seeded workloads.
+
+Codes and scale bits must be identical; attention outputs (bf16) must be within
+max-abs 2e-2 and mean-abs 2e-3 of the fp64 oracle evaluated on the same codes.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import slim_oracle as so
+from paper_2407_07304_b200 import workloads
+from helpers import bf16_bits
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 2e-2
+MEAN_ABS = 2e-3
+
+
+def _oracle_cache(w):
+    """Oracle codes/scales of every sequence's K and V (all rows the run appends)."""
+    out = []
+    for b in range(w.B):
+        kc, ks = so.quantize(bf16_bits(w.k[b]))
+        vc, vs = so.quantize(bf16_bits(w.v[b]))
+        out.append((kc, ks, vc, vs))
+    return out
+
+
+def _assert_cache_bits(run, oc):
+    for b in range(run.w.B):
+        kc, ks, vc, vs = run.gather_cache(b)
+        T = run.pos[b]
+        assert np.array_equal(kc.numpy(), oc[b][0][:T]), f"K codes differ (seq {b})"
+        assert np.array_equal(vc.numpy(), oc[b][2][:T]), f"V codes differ (seq {b})"
+        assert np.array_equal(ks.numpy().view(np.uint32), oc[b][1][:T].view(np.uint32)), f"K scales differ (seq {b})"
+        assert np.array_equal(vs.numpy().view(np.uint32), oc[b][3][:T].view(np.uint32)), f"V scales differ (seq {b})"
+
+
+def _assert_close(got_bf16, want_f64, what):
+    got = got_bf16.float().cpu().numpy().astype(np.float64)
+    err = np.abs(got - want_f64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    assert err.max() <= MAX_ABS, f"{what}: max-abs {err.max():.3e}"
+    assert err.mean() <= MEAN_ABS, f"{what}: mean-abs {err.mean():.3e}"
+    return err.max(), err.mean()
+
+
+def _sample_rows(n, extra, seed):
+    base = [r for r in (0, 1, 63, 64, 65, 127, 128, 129, n - 2, n - 1) if 0 <= r < n]
+    rng = np.random.default_rng(seed)
+    more = rng.integers(0, n, size=extra).tolist() if n > len(base) else []
+    return sorted(set(base + more))
+
+
+def _check(w, prefill_rows=None, decode_steps=None):
+    """Run the workload on the GPU and compare everything (or the given samples) with the oracle."""
+    from paper_2407_07304_b200 import harness
+    oc = _oracle_cache(w)
+    run, out_prefill, outs = harness.run_workload(w, decode_steps=decode_steps)
+    _assert_cache_bits(run, oc)
+    if out_prefill is not None:
+        for b in range(w.B):
+            n = w.prefill_len[b]
+            sel = None if prefill_rows is None else _sample_rows(n, prefill_rows, 17 + b)
+            want = so.attention(bf16_bits(w.q_prefill[b]), oc[b][0], oc[b][1], oc[b][2], oc[b][3], n, w.sm_scale, sel=sel)
+            got = out_prefill[b] if sel is None else out_prefill[b][torch.tensor(sel, device=out_prefill[b].device)]
+            _assert_close(got, want, f"{w.name} prefill seq {b}")
+    for s, o in outs.items():
+        for b in range(w.B):
+            L = w.prefill_len[b] + w.bulk_len[b] + s + 1
+            want = so.attention(bf16_bits(w.q_decode[s, b:b + 1]), oc[b][0], oc[b][1], oc[b][2], oc[b][3], L, w.sm_scale)
+            _assert_close(o[b:b + 1], want, f"{w.name} decode step {s} seq {b}")
+
+
+# ---------------------------------------------------------------- small versions: every output compared
+@pytest.mark.parametrize("index,shrink", [(1, 1), (2, 8), (3, 16), (4, 8), (5, 32)])
+def test_workload_small_all_outputs(index, shrink):
+    _check(workloads.make_workload(index, shrink=shrink))
+
+
+# ---------------------------------------------------------------- full sizes
+def test_c2_full_all_rows():
+    _check(workloads.make_workload(2))
+
+
+def test_c4_full_all_rows():
+    _check(workloads.make_workload(4))
+
+
+def test_c3_full_sampled_rows():
+    _check(workloads.make_workload(3), prefill_rows=48)
+
+
+def test_c5_full_sampled():
+    _check(workloads.make_workload(5), prefill_rows=24, decode_steps={0, 31, 63})
+
+
+# ---------------------------------------------------------------- edge cases
+def _custom(B, Hq, Hkv, prefill, bulk, steps, seed):
+    g = torch.Generator().manual_seed(seed)
+    w = workloads.Workload(f"custom{seed}", 0, B, Hq, Hkv, prefill, bulk, steps)
+    for b in range(B):
+        T = w.total_len(b)
+        w.k.append(torch.randn((T, Hkv, 128), generator=g).to(torch.bfloat16))
+        w.v.append(torch.randn((T, Hkv, 128), generator=g).to(torch.bfloat16))
+    if any(prefill):
+        w.q_prefill = [torch.randn((n, Hq, 128), generator=g).to(torch.bfloat16) for n in prefill]
+    if steps:
+        w.q_decode = torch.randn((steps, B, Hq, 128), generator=g).to(torch.bfloat16)
+    return w
+
+
+@pytest.mark.parametrize("lens", [[1], [2, 127], [128, 129], [255, 256, 257], [1, 383, 640]])
+def test_ragged_lengths_prefill_and_decode(lens):
+    B = len(lens)
+    _check(_custom(B, 4, 2, lens, [0] * B, 2, 100 + lens[0]))
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(1, 1), (8, 1), (16, 1), (12, 3), (6, 2)])
+def test_group_sizes(Hq, Hkv):
+    _check(_custom(2, Hq, Hkv, [70, 200], [37, 0], 2, 200 + Hq))
+
+
+def test_scale_extremes_and_zero_rows():
+    # rows scaled far apart, zero K and V rows, and large-magnitude queries
+    w = _custom(1, 2, 1, [150], [0], 2, 300)
+    w.k[0][5] = 0
+    w.v[0][7] = 0
+    w.v[0][20:40] *= 2.0 ** -12
+    w.v[0][60:70] *= 2.0 ** 10
+    w.k[0][80:90] *= 2.0 ** -9
+    w.q_prefill[0][100:110] *= 64.0
+    w.q_decode[0] *= 2.0 ** -8
+    oc = _oracle_cache(w)
+    from paper_2407_07304_b200 import harness
+    run, out_prefill, outs = harness.run_workload(w)
+    _assert_cache_bits(run, oc)
+    want = so.attention(bf16_bits(w.q_prefill[0]), *oc[0], 150, w.sm_scale)
+    got = out_prefill[0].float().cpu().numpy().astype(np.float64)
+    # outputs span 2^10: compare relative to each row's magnitude
+    denom = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - want) / denom).max() < 2e-2
+    for s, o in outs.items():
+        want = so.attention(bf16_bits(w.q_decode[s]), *oc[0], 151 + s, w.sm_scale)
+        denom = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
+        assert (np.abs(o.float().cpu().numpy() - want) / denom).max() < 2e-2
+
+
+def test_chunked_prefill_offset_and_shuffled_pages():
+    # q_len < kv_len (the last 50 of 300 cached tokens attend) through a permuted block table
+    from paper_2407_07304_b200 import harness
+    w = _custom(2, 4, 2, [300, 140], [0, 0], 0, 400)
+    pages = w.pages_per_seq()
+    perm = torch.randperm(2 * pages + 3, generator=torch.Generator().manual_seed(1))[:2 * pages]
+    bt = perm.to(torch.int32).view(2, pages)
+    run = harness.LayerRun(w, block_table=bt, num_pages=2 * pages + 3)
+    run.append(w.prefill_len)
+    oc = _oracle_cache(w)
+    _assert_cache_bits(run, oc)
+    tails = [50, 140]
+    outs = run.prefill([w.q_prefill[b][-tails[b]:] for b in range(2)])
+    torch.cuda.synchronize()
+    for b in range(2):
+        want = so.attention(bf16_bits(w.q_prefill[b][-tails[b]:]), *oc[b], w.prefill_len[b], w.sm_scale)
+        _assert_close(outs[b], want, f"chunked prefill seq {b}")
+
+
+def test_empty_and_zero_length():
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = _custom(2, 2, 1, [0, 0], [0, 5], 0, 500)
+    run = harness.LayerRun(w)
+    run.append([0, 5])
+    q = torch.randn((2, 2, 128)).to(torch.bfloat16)
+    out = run.decode(q)
+    torch.cuda.synchronize()
+    assert not out[0].any()            # kv_len 0 -> zeros
+    oc = _oracle_cache(w)
+    want = so.attention(bf16_bits(q[1:2]), *oc[1], 5, w.sm_scale)
+    _assert_close(out[1:2], want, "short decode")
+    # B == 0 and max_new == 0 are no-ops
+    slim.slim_kv_append(run.cache, None, None, None, None, 0, 0)
+    slim.slim_attn_decode(run.cache, None, None, None, 0, 0, 2, 1.0, run.ws_decode)
+
+
+def test_bad_arguments_are_rejected_on_the_host():
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = _custom(1, 4, 2, [0], [10], 0, 600)
+    run = harness.LayerRun(w)
+    q = torch.zeros((1, 4, 128), dtype=torch.bfloat16, device="cuda")
+    kvl = torch.tensor([10], dtype=torch.int32, device="cuda")
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_attn_decode(run.cache, q, q.clone(), kvl, 1, 10, 3, 1.0, run.ws_decode)   # 3 % 2 != 0
+    assert e.value.code == slim.SLIM_ERR_UNSUPPORTED
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_attn_decode(run.cache, q, q.clone(), kvl, 1, 10, 4, 1.0, None)
+    assert e.value.code == slim.SLIM_ERR_WORKSPACE
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_attn_decode(run.cache, None, q, kvl, 1, 10, 4, 1.0, run.ws_decode)
+    assert e.value.code == slim.SLIM_ERR_INVALID_ARG
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_attn_decode(run.cache, q, q.clone(), kvl, 1, 100000, 4, 1.0, run.ws_decode)  # beyond the page table
+    assert e.value.code == slim.SLIM_ERR_INVALID_ARG
+    torch.cuda.synchronize()
