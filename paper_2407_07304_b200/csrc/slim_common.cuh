@@ -117,6 +117,19 @@ __device__ __forceinline__ float pow2_recip(float p2)
     return __uint_as_float((uint32_t)(254 - e) << 23);
 }
 
+// log2 and reciprocal of a V scale.  A zero scale (all-zero row, codes all zero) is
+// replaced by 2^-100: the row then adds nothing to the numerator and its softmax
+// weight still reaches the denominator.
+constexpr float kMinScale = 7.888609052210118e-31f;   // 2^-100
+__device__ __forceinline__ float log2_scale(float sv)
+{
+    return __log2f(fmaxf(sv, kMinScale));
+}
+__device__ __forceinline__ float recip_scale(float sv)
+{
+    return __frcp_rn(fmaxf(sv, kMinScale));
+}
+
 __device__ __forceinline__ float warp_max(float v)
 {
 #pragma unroll

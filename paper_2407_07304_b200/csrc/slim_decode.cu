@@ -10,6 +10,13 @@
 // rescale.  The G = Hq / Hkv query heads that share the kv head form the rows of
 // a 16-row tensor-core tile, so each cached byte is converted and used once for
 // all of them.
+//
+// The V scale of key j is folded into the softmax weight: with
+//   s'_j = s_j + log2(scale_v[j]),  m' = max_j s'_j,  P_j = 2^(s'_j - m')
+// the output is  o = (sum_j P_j * v_code_j) / (sum_j P_j / scale_v[j]),
+// identical to softmax(s) . (v_code * scale_v) because the factor 2^(-m') cancels.
+// P_j <= 1 is normalised by the row's largest contribution, which is what makes
+// its fp16 copy for the tensor cores safe whatever the spread of the V scales.
 #include "slim_common.cuh"
 
 namespace slim {
@@ -114,16 +121,18 @@ slim_decode_split_kernel(const DecodeParams p)
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
             qk_tile(acc, qf, kbuf, tok0, g, t);
             const float2 sk = *reinterpret_cast<const float2 *>(ksc + tok0 + 2 * t);
+            const float2 sv = *reinterpret_cast<const float2 *>(vsc + tok0 + 2 * t);
+            const float lx = log2_scale(sv.x), ly = log2_scale(sv.y);
             if (ROWS == 1) {
                 if (g == 0)
                     *reinterpret_cast<float2 *>(S + tok0 + 2 * t) =
-                        make_float2(acc[0] * sk.x * rs_lo, acc[1] * sk.y * rs_lo);
+                        make_float2(fmaf(acc[0], sk.x * rs_lo, lx), fmaf(acc[1], sk.y * rs_lo, ly));
             } else {
                 *reinterpret_cast<float2 *>(S + g * C + tok0 + 2 * t) =
-                    make_float2(acc[0] * sk.x * rs_lo, acc[1] * sk.y * rs_lo);
+                    make_float2(fmaf(acc[0], sk.x * rs_lo, lx), fmaf(acc[1], sk.y * rs_lo, ly));
                 if (ROWS > 8)
                     *reinterpret_cast<float2 *>(S + (g + 8) * C + tok0 + 2 * t) =
-                        make_float2(acc[2] * sk.x * rs_hi, acc[3] * sk.y * rs_hi);
+                        make_float2(fmaf(acc[2], sk.x * rs_hi, lx), fmaf(acc[3], sk.y * rs_hi, ly));
             }
         }
     };
@@ -141,12 +150,7 @@ slim_decode_split_kernel(const DecodeParams p)
     }
     __syncthreads();
 
-    // ---- one softmax per row over the chunk; P = exp2(s - m) * scale_v / vp2 in fp16,
-    //      vp2 a power of two near the chunk's largest V scale (keeps P in fp16 range)
-    float vmax = 0.f;
-    for (int i = lane; i < n_tok; i += 32) vmax = fmaxf(vmax, vsc[i]);
-    const float vp2 = pow2_floor(warp_max(vmax));
-    const float vinv = pow2_recip(vp2);
+    // ---- one softmax per row over the chunk: P = 2^(s' - m') in fp16, l = sum P / scale_v in fp32
     const int n_pad = (n_tok + 15) & ~15;
     for (int r = warp; r < ROWS; r += 4) {
         if (r >= p.G) break;
@@ -155,13 +159,12 @@ slim_decode_split_kernel(const DecodeParams p)
         m = warp_max(m);
         float l = 0.f;
         for (int i = lane; i < n_pad; i += 32) {
-            float e = 0.f, pv = 0.f;
+            float e = 0.f;
             if (i < n_tok) {
                 e = exp2f(S[r * C + i] - m);
-                pv = e * (vsc[i] * vinv);
+                l = fmaf(e, recip_scale(vsc[i]), l);
             }
-            l += e;
-            P[r * L::PSTRIDE + i] = __float2half_rn(pv);
+            P[r * L::PSTRIDE + i] = __float2half_rn(e);
         }
         l = warp_sum(l);
         if (lane == 0) {
@@ -227,13 +230,13 @@ slim_decode_split_kernel(const DecodeParams p)
     const int d0 = 32 * warp + 8 * t;
     if (g < p.G) {
         float *dst = p.part_o + (((size_t)b * p.Hq + h0 + g) * p.n_chunks + chunk) * kHeadDim + d0;
-        *reinterpret_cast<float4 *>(dst) = make_float4(o[0][0] * vp2, o[1][0] * vp2, o[2][0] * vp2, o[3][0] * vp2);
-        *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[0][1] * vp2, o[1][1] * vp2, o[2][1] * vp2, o[3][1] * vp2);
+        *reinterpret_cast<float4 *>(dst) = make_float4(o[0][0], o[1][0], o[2][0], o[3][0]);
+        *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[0][1], o[1][1], o[2][1], o[3][1]);
     }
     if (ROWS > 8 && g + 8 < p.G) {
         float *dst = p.part_o + (((size_t)b * p.Hq + h0 + g + 8) * p.n_chunks + chunk) * kHeadDim + d0;
-        *reinterpret_cast<float4 *>(dst) = make_float4(o[0][2] * vp2, o[1][2] * vp2, o[2][2] * vp2, o[3][2] * vp2);
-        *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[0][3] * vp2, o[1][3] * vp2, o[2][3] * vp2, o[3][3] * vp2);
+        *reinterpret_cast<float4 *>(dst) = make_float4(o[0][2], o[1][2], o[2][2], o[3][2]);
+        *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[0][3], o[1][3], o[2][3], o[3][3]);
     }
 }
 

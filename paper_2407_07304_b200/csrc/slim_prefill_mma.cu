@@ -8,6 +8,11 @@
 // softmax attention.  INT8 tiles arrive by 16-byte asynchronous copies, are
 // converted to fp16 in registers (Section 2.2 hybrid-dtype step) and feed
 // mma.sync tensor-core tiles.
+//
+// The V scale of key j is folded into the softmax weight: with
+//   s'_j = s_j + log2(scale_v[j]),  m' = running max of s',  P_j = 2^(s'_j - m')
+// the output is  o = (sum_j P_j * v_code_j) / (sum_j P_j / scale_v[j]),
+// identical to softmax(s) . (v_code * scale_v) because the factor 2^(-m') cancels.
 #include "slim_common.cuh"
 
 namespace slim {
@@ -91,7 +96,6 @@ slim_prefill_mma_kernel(const PrefillParams p)
 #pragma unroll
         for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-    float kr = pow2_floor(0.f);   // running power-of-two normaliser of the V scales (starts at the floor)
 
     for (int kt = 0; kt < n_tiles; ++kt) {
         if (kt + 1 < n_tiles) {
@@ -117,22 +121,18 @@ slim_prefill_mma_kernel(const PrefillParams p)
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
             const float2 sk = *reinterpret_cast<const float2 *>(st.ks + nt * 8 + 2 * t);
+            const float2 sv = *reinterpret_cast<const float2 *>(st.vs + nt * 8 + 2 * t);
+            const float lsv[2] = {log2_scale(sv.x), log2_scale(sv.y)};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int key = tok0 + nt * 8 + 2 * t + (j & 1);
                 const int r = j >> 1;
-                const float v = s[nt][j] * ((j & 1) ? sk.y : sk.x) * rs[r];
+                const float v = fmaf(s[nt][j], ((j & 1) ? sk.y : sk.x) * rs[r], lsv[j & 1]);
                 s[nt][j] = (key <= last_key[r] && key < n_keys) ? v : -INFINITY;
                 mx[r] = fmaxf(mx[r], s[nt][j]);
             }
         }
-        // ---- running maximum, V-scale normaliser and rescale of the accumulators
-        float vmax = 0.f;
-        for (int i = lane; i < rows; i += 32) vmax = fmaxf(vmax, st.vs[i]);
-        const float kr_new = fmaxf(kr, pow2_floor(warp_max(vmax)));
-        const float kr_ratio = kr * pow2_recip(kr_new);
-        const float kinv = pow2_recip(kr_new);
-        kr = kr_new;
+        // ---- running maximum and rescale of the accumulators
         float msafe[2];
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
@@ -143,14 +143,13 @@ slim_prefill_mma_kernel(const PrefillParams p)
             const float corr = exp2f(m_run[r] - msafe[r]);
             m_run[r] = m_new;
             l_run[r] *= corr;
-            const float oc = corr * kr_ratio;
 #pragma unroll
             for (int nd = 0; nd < 16; ++nd) {
-                o[nd][2 * r] *= oc;
-                o[nd][2 * r + 1] *= oc;
+                o[nd][2 * r] *= corr;
+                o[nd][2 * r + 1] *= corr;
             }
         }
-        // ---- P = exp2(s - m) (row sums in fp32), times the V scale, to fp16 A-fragments
+        // ---- P = 2^(s' - m') to fp16 A-fragments; l += P / scale_v in fp32
         uint32_t pa[4][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
@@ -160,9 +159,8 @@ slim_prefill_mma_kernel(const PrefillParams p)
             for (int j = 0; j < 4; ++j) {
                 const int r = j >> 1;
                 const bool vis = s[nt][j] != -INFINITY;
-                const float e = vis ? exp2f(s[nt][j] - msafe[r]) : 0.f;
-                l_run[r] += e;
-                pv[j] = vis ? e * (((j & 1) ? sv.y : sv.x) * kinv) : 0.f;
+                pv[j] = vis ? exp2f(s[nt][j] - msafe[r]) : 0.f;
+                if (vis) l_run[r] = fmaf(pv[j], recip_scale((j & 1) ? sv.y : sv.x), l_run[r]);
             }
             pa[nt >> 1][(nt & 1) * 2 + 0] = pack_half2(pv[0], pv[1]);
             pa[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(pv[2], pv[3]);
@@ -203,7 +201,7 @@ slim_prefill_mma_kernel(const PrefillParams p)
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
         if (row >= q_len) continue;
-        const float f = (l > 0.f) ? kr / l : 0.f;
+        const float f = (l > 0.f) ? 1.f / l : 0.f;
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
