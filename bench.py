@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the SlimAttention / INT8 KV cache hot path on B200.
+
+One step = one pass of the decode hot path on the Llama-2-7B-shaped workload
+(batch 16, 32 q = 32 kv heads, head_dim 128, 2048 cached tokens + 1 new token
+per sequence): quantise-and-append the new K/V rows, then split + merge decode
+attention over the 2049-token INT8 cache.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (under torchrun) every rank runs the same per-GPU workload on its own
+GPU (sequences are independent; no collective on the data path; weak scaling)
+and the line reports the aggregate over ranks with the max-over-ranks time.
+`--impl reference` times the CPU oracle on the host cores instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode attention tokens/s (append + split/merge decode over the INT8 KV cache)"
+UNIT = "tokens/s"
+ROW_BYTES = 264            # per (token, kv head): 128 K codes + 128 V codes + 2 fp32 scales
+N_ROT = 3                  # independent cache copies rotated between steps (3 x 277 MB >> 126 MB L2)
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops", 1590.0)), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle sampling while the timed region runs (read-only queries)."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.gpu_index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, sm_max, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                sm_max.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(sm_max) if sm_max else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places this file touches oracle/)
+# ---------------------------------------------------------------------------------------------
+def _bits(t):
+    import numpy as np
+    import torch
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+class OracleStep:
+    """The decode step of the workload on the CPU oracle, on the first n_seq sequences."""
+
+    def __init__(self, w, n_seq):
+        from oracle import slim_oracle as so
+        self.so, self.w, self.n_seq = so, w, n_seq
+        self.ctx = w.bulk_len[0]
+        self.cache = []
+        for b in range(n_seq):
+            kc, ks = so.quantize(_bits(w.k[b]))
+            vc, vs = so.quantize(_bits(w.v[b]))
+            self.cache.append([kc, ks, vc, vs])
+        self.k_new = [_bits(w.k[b][self.ctx:self.ctx + 1]) for b in range(n_seq)]
+        self.v_new = [_bits(w.v[b][self.ctx:self.ctx + 1]) for b in range(n_seq)]
+        self.q = [_bits(w.q_decode[0, b:b + 1]) for b in range(n_seq)]
+
+    def step(self):
+        so, c = self.so, self.ctx
+        for b in range(self.n_seq):
+            kc, ks, vc, vs = self.cache[b]
+            kc[c:c + 1], ks[c:c + 1] = so.quantize(self.k_new[b])
+            vc[c:c + 1], vs[c:c + 1] = so.quantize(self.v_new[b])
+            so.attention(self.q[b], kc, ks, vc, vs, c + 1, self.w.sm_scale)
+
+
+def cpu_baseline(w, budget_s=12.0, max_reps=100):
+    from oracle import slim_oracle as so
+    st = OracleStep(w, w.B)
+    st.step()
+    reps, t0 = 0, time.perf_counter()
+    while reps < max_reps and time.perf_counter() - t0 < budget_s:
+        st.step()
+        reps += 1
+    dt = time.perf_counter() - t0
+    return {"value": w.B * reps / dt, "unit": UNIT, "cores": so.threads(), "kind": "oracle",
+            "sample": f"all {w.B} sequences of the workload, full step (quantise new rows + fp64 attention over "
+                      f"{st.ctx + 1} tokens), {reps} repetitions in {dt:.1f} s"}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    from oracle import slim_oracle as so
+    from paper_2407_07304_b200 import workloads
+    w = workloads.make_workload(2)
+    n_seq = 2                                    # bounded sample: 2 of the 16 sequences per step
+    st = OracleStep(w, n_seq)
+    for _ in range(args.warmup):
+        st.step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        st.step()
+    dt = time.perf_counter() - t0
+    value = n_seq * args.steps / dt
+    sample = f"{n_seq} of {w.B} sequences per step (all 32 heads, {st.ctx + 1} tokens), fp64 CPU oracle as it stands"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": 128,
+                   "context": st.ctx + 1, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": so.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+# CUDA arm
+# ---------------------------------------------------------------------------------------------
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_07304_b200 import binding as slim, workloads
+    from paper_2407_07304_b200.harness import LayerRun
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the attention path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = workloads.make_workload(2)
+    B, Hq, Hkv, ctx = w.B, w.Hq, w.Hkv, w.bulk_len[0]
+    kv_len_host = [ctx + 1] * B
+
+    # N_ROT independent caches, each pre-filled (untimed) with the 2048-token context
+    runs = []
+    for _ in range(N_ROT):
+        r = LayerRun(w, device=dev)
+        r.append(w.bulk_len)
+        runs.append(r)
+    torch.cuda.synchronize()
+    k_new = torch.cat([w.k[b][ctx:ctx + 1] for b in range(B)]).to(dev).contiguous()    # [B, Hkv, 128]
+    v_new = torch.cat([w.v[b][ctx:ctx + 1] for b in range(B)]).to(dev).contiguous()
+    q = w.q_decode[0].to(dev).contiguous()
+    out = torch.empty_like(q)
+    cu_new = torch.arange(B + 1, dtype=torch.int32, device=dev)
+    start_pos = torch.full((B,), ctx, dtype=torch.int32, device=dev)
+    kv_len = torch.full((B,), ctx + 1, dtype=torch.int32, device=dev)
+    max_kv = ctx + 1
+    ws = runs[0].ws_decode
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        c = runs[i % N_ROT].cache
+        slim.slim_kv_append(c, k_new, v_new, cu_new, start_pos, B, 1, stream)
+        slim.slim_attn_decode(c, q, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        barrier()
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.1)
+    # ---- headline: device-resident inputs, whole step
+    ms_total = timed(step, args.steps)
+    # ---- per-kernel: the split kernel alone, events around every launch
+    split_ms = []
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        c = runs[i % N_ROT].cache
+        slim.slim_kv_append(c, k_new, v_new, cu_new, start_pos, B, 1, stream)
+        evs[i][0].record(stream)
+        slim.slim_attn_decode_split(c, q, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
+        evs[i][1].record(stream)
+        slim.slim_attn_decode_merge(c, out, kv_len, B, max_kv, Hq, ws, stream)
+    torch.cuda.synchronize()
+    split_ms = [a.elapsed_time(b) for a, b in evs]
+    # ---- end to end: host (pinned) inputs and outputs through slim_decode_step_host
+    q_h, k_h, v_h = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+    out_h = torch.empty_like(q_h).pin_memory()
+    staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
+
+    def step_host(i):
+        c = runs[i % N_ROT].cache
+        slim.slim_decode_step_host(c, q_h, k_h, v_h, out_h, staging, cu_new, start_pos, kv_len, B, max_kv, Hq,
+                                   w.sm_scale, ws, stream)
+        stream.synchronize()        # the caller needs the result before the next token
+
+    for i in range(3):
+        step_host(i)
+    ms_e2e = timed(step_host, args.steps)
+    clocks = sampler.stop() if sampler else None
+    same = torch.equal(out_h, out.cpu())
+
+    # ---- extra single-GPU context numbers (not part of the headline): prefill of workload 3
+    extra = {}
+    if rank == 0 and world == 1 and not args.no_extra:
+        extra = extra_numbers(slim, workloads, dev)
+
+    if rank != 0:
+        return
+    hbm_peak, bf16_peak, peak_kind = _peaks()
+    tokens = world * B * args.steps
+    cache_bytes = sum(kv_len_host) * Hkv * ROW_BYTES
+    split_bytes = cache_bytes + B * Hq * 128 * 2
+    # whole step: cache read once, Q in, O out, new K/V rows read as bf16 and written as codes + scales
+    step_bytes = cache_bytes + 2 * B * Hq * 256 + B * Hkv * (2 * 256 + ROW_BYTES)
+    split_avg_ms = statistics.mean(split_ms)
+    achieved = split_bytes / (split_avg_ms * 1e-3) / 1e9
+    h2d = (B * Hq + 2 * B * Hkv) * 128 * 2
+    d2h = B * Hq * 128 * 2
+    line = {
+        "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 mma, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
+                   "context": ctx + 1, "cache": "int8 codes + fp32 scale per (token, kv head), 128-token pages",
+                   "l2": f"inputs larger than L2: {N_ROT} cache copies of {cache_bytes / 1e6:.0f} MB rotated",
+                   "parallelism": f"dp{world} (independent sequences per GPU, no collective)"},
+        "hbm_gbs_step_per_gpu": step_bytes / (ms_total / args.steps * 1e-3) / 1e9,
+        "pct_of_8tbs_step": 100.0 * step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / 8000.0,
+        "roofline": {"bound": "hbm", "kernel": "slim_decode_split_kernel", "achieved": achieved, "peak": hbm_peak,
+                     "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_8tbs": achieved / 8000.0, "bytes_per_launch": split_bytes,
+                     "avg_launch_ms": split_avg_ms, "min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same)},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu:
+        line["cpu_baseline"] = cpu_baseline(w)
+    if extra:
+        line["extra"] = extra
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram bytes read + written by one slim_decode_split_kernel launch on this workload, from the ncu
+# capture summarised under profiles/ ; None until a capture of the current kernel exists.
+TRAFFIC_PER_LAUNCH = None
+
+
+def extra_numbers(slim, workloads, dev):
+    """Prefill of workload 3 (S = 8192) timed alone: TFLOP/s against the bf16 dense peak."""
+    import torch
+    from paper_2407_07304_b200.harness import LayerRun
+    _, bf16_peak, peak_kind = _peaks()
+    w3 = workloads.make_workload(3)
+    run = LayerRun(w3, device=dev)
+    S = w3.prefill_len[0]
+    k_new, v_new = run.k[0].contiguous(), run.v[0].contiguous()
+    cu = torch.tensor([0, S], dtype=torch.int32, device=dev)
+    zero = torch.zeros(1, dtype=torch.int32, device=dev)
+    kvl = torch.tensor([S], dtype=torch.int32, device=dev)
+    q = w3.q_prefill[0].to(dev).contiguous()
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+
+    def append():
+        slim.slim_kv_append(run.cache, k_new, v_new, cu, zero, 1, S, stream)
+
+    def prefill():
+        slim.slim_attn_prefill(run.cache, q, out, cu, kvl, 1, S, S, w3.Hq, w3.sm_scale, run.ws_prefill, stream)
+
+    def time_it(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms_append = time_it(append, 20)
+    ms_prefill = time_it(prefill, 5)
+    flops = 4 * 128 * w3.Hq * S * (S + 1) // 2
+    append_bytes = S * w3.Hkv * (2 * 256 + ROW_BYTES)
+    hbm_peak, _, _ = _peaks()
+    return {
+        "prefill_c3": {"workload": w3.name, "ms": ms_prefill, "tflops": flops / (ms_prefill * 1e-3) / 1e12,
+                       "frac_of_bf16_peak": flops / (ms_prefill * 1e-3) / 1e12 / bf16_peak,
+                       "peak_tflops": bf16_peak, "peak_kind": f"of {peak_kind}",
+                       "tokens_per_s_with_append": S / ((ms_prefill + ms_append) * 1e-3)},
+        "append_c3": {"ms": ms_append, "gbs": append_bytes / (ms_append * 1e-3) / 1e9,
+                      "frac_of_hbm_peak": append_bytes / (ms_append * 1e-3) / 1e9 / hbm_peak},
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=30)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-extra", action="store_true", help="skip the prefill context numbers")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -143,6 +143,45 @@ int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out,
                      const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * The two passes of slim_attn_decode as separate calls, for callers that schedule
+ * or time them individually: the split pass (every block: the scores of its key
+ * chunk, one softmax over the chunk, the product with V; Section 2.1 order inside
+ * the chunk) writes partials into `workspace`; the merge pass combines them into
+ * `out`.  Same arguments, validation and workspace as slim_attn_decode;
+ * slim_attn_decode(...) == split(...) followed by merge(...) on the same stream.
+ */
+int slim_attn_decode_split(const slim_cache_t *cache, const void *q,
+                           const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                           void *workspace, size_t workspace_bytes, void *stream);
+int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
+                           const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq,
+                           const void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * One decode step from host buffers: copies the step's query and new K/V rows
+ * (one new token per sequence) host -> device, appends them (slim_kv_append),
+ * runs slim_attn_decode over the lengthened cache and copies the result device
+ * -> host, all asynchronously on `stream` (Section 2.2: the per-token step whose
+ * cache traffic Eq. 1 counts).  Host buffers should be pinned; they must stay
+ * valid and out_host must not be read until the stream has been synchronised.
+ *
+ *   q_host      host bf16 [B][Hq][128]
+ *   k_new_host, v_new_host  host bf16 [B][num_kv_heads][128]
+ *   out_host    host bf16 [B][Hq][128]
+ *   staging     device scratch of at least slim_step_staging_bytes(B, Hq, Hkv) bytes, 16-byte aligned
+ *   cu_new      device int32 [B+1] = 0, 1, ..., B
+ *   start_pos   device int32 [B]: position the new token of sequence b is written to
+ *   kv_len      device int32 [B]: cached tokens per sequence after the append (start_pos + 1)
+ *   workspace   as for slim_attn_decode
+ */
+int slim_decode_step_host(const slim_cache_t *cache, const void *q_host, const void *k_new_host,
+                          const void *v_new_host, void *out_host, void *staging, size_t staging_bytes,
+                          const int32_t *cu_new, const int32_t *start_pos, const int32_t *kv_len,
+                          int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                          void *workspace, size_t workspace_bytes, void *stream);
+size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
+
 /* Scratch bytes needed by a phase (SLIM_PHASE_*) for the given shape; 0 on invalid arguments. */
 size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q, int32_t max_kv);
 

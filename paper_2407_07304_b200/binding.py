@@ -24,7 +24,8 @@ HEAD_DIM = 128
 PAGE_TOKENS = 128
 
 EXPORTS = (
-    "slim_kv_append", "slim_attn_prefill", "slim_attn_decode", "slim_workspace_bytes",
+    "slim_kv_append", "slim_attn_prefill", "slim_attn_decode", "slim_attn_decode_split",
+    "slim_attn_decode_merge", "slim_decode_step_host", "slim_step_staging_bytes", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -73,6 +74,14 @@ def lib():
         L.slim_attn_prefill.restype = ctypes.c_int
         L.slim_attn_decode.argtypes = [CP, P, P, P, I, I, I, F, P, Z, P]
         L.slim_attn_decode.restype = ctypes.c_int
+        L.slim_attn_decode_split.argtypes = [CP, P, P, I, I, I, F, P, Z, P]
+        L.slim_attn_decode_split.restype = ctypes.c_int
+        L.slim_attn_decode_merge.argtypes = [CP, P, P, I, I, I, P, Z, P]
+        L.slim_attn_decode_merge.restype = ctypes.c_int
+        L.slim_decode_step_host.argtypes = [CP, P, P, P, P, P, Z, P, P, P, I, I, I, F, P, Z, P]
+        L.slim_decode_step_host.restype = ctypes.c_int
+        L.slim_step_staging_bytes.argtypes = [I, I, I]
+        L.slim_step_staging_bytes.restype = Z
         L.slim_workspace_bytes.argtypes = [I, I, I, I, I, I]
         L.slim_workspace_bytes.restype = Z
         L.slim_cache_code_bytes.argtypes = [I, I]
@@ -91,6 +100,10 @@ def lib():
 
 def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _nbytes(t):
+    return 0 if t is None else t.numel() * t.element_size()
 
 
 def _stream(stream):
@@ -151,6 +164,32 @@ def slim_attn_decode(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, workspace, 
     rc = lib().slim_attn_decode(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(kv_len), B, max_kv, Hq,
                                 sm_scale, _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "slim_attn_decode")
+
+
+def slim_attn_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None):
+    rc = lib().slim_attn_decode_split(ctypes.byref(cache.struct), _ptr(q), _ptr(kv_len), B, max_kv, Hq, sm_scale,
+                                      _ptr(workspace), _nbytes(workspace), _stream(stream))
+    _check(rc, "slim_attn_decode_split")
+
+
+def slim_attn_decode_merge(cache, out, kv_len, B, max_kv, Hq, workspace, stream=None):
+    rc = lib().slim_attn_decode_merge(ctypes.byref(cache.struct), _ptr(out), _ptr(kv_len), B, max_kv, Hq,
+                                      _ptr(workspace), _nbytes(workspace), _stream(stream))
+    _check(rc, "slim_attn_decode_merge")
+
+
+def slim_decode_step_host(cache, q_host, k_new_host, v_new_host, out_host, staging, cu_new, start_pos, kv_len,
+                          B, max_kv, Hq, sm_scale, workspace, stream=None):
+    """q_host / k_new_host / v_new_host / out_host are CPU (pinned) bf16 tensors."""
+    rc = lib().slim_decode_step_host(ctypes.byref(cache.struct), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host),
+                                     _ptr(out_host), _ptr(staging), _nbytes(staging), _ptr(cu_new), _ptr(start_pos),
+                                     _ptr(kv_len), B, max_kv, Hq, sm_scale, _ptr(workspace), _nbytes(workspace),
+                                     _stream(stream))
+    _check(rc, "slim_decode_step_host")
+
+
+def slim_step_staging_bytes(B, Hq, Hkv):
+    return lib().slim_step_staging_bytes(B, Hq, Hkv)
 
 
 def slim_workspace_bytes(phase, B, Hq, Hkv, max_q, max_kv):

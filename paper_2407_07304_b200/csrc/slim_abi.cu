@@ -15,8 +15,10 @@ int set_cuda_error(cudaError_t e)
 
 int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
                   const int32_t *start_pos, int B, int max_new, cudaStream_t stream);
-int launch_decode(const slim_cache_t *c, const void *q, void *out, const int32_t *kv_len, int B, int max_kv,
-                  int Hq, float sm_scale, void *workspace, cudaStream_t stream);
+int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv, int Hq,
+                        float sm_scale, void *workspace, cudaStream_t stream);
+int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
+                        const void *workspace, cudaStream_t stream);
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_mma(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                        int B, int max_q, int Hq, float sm_scale, cudaStream_t stream);
@@ -67,23 +69,96 @@ SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void
     return launch_prefill_mma(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, (cudaStream_t)stream);
 }
 
-SLIM_EXPORT int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out, const int32_t *kv_len,
-                                 int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
-                                 size_t workspace_bytes, void *stream)
+// Shared validation of the decode entry points; *launch is false for a valid no-op.
+static int check_decode(const slim_cache_t *cache, int32_t B, int32_t max_kv, int32_t Hq, const void *workspace,
+                        size_t workspace_bytes, bool *launch)
 {
+    *launch = false;
     int rc = check_cache(cache);
     if (rc != SLIM_OK) return rc;
     if (B < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
     if (Hq % cache->num_kv_heads != 0 || Hq / cache->num_kv_heads > 16) return SLIM_ERR_UNSUPPORTED;
     if (B == 0) return SLIM_OK;
-    if (q == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
-    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
     if (B > 65535 || cache->num_kv_heads > 65535) return SLIM_ERR_UNSUPPORTED;
     if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
     const size_t need = slim_workspace_bytes(SLIM_PHASE_DECODE, B, Hq, cache->num_kv_heads, 1, max_kv);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
     if ((uintptr_t)workspace & 15) return SLIM_ERR_INVALID_ARG;
-    return launch_decode(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+    *launch = true;
+    return SLIM_OK;
+}
+
+SLIM_EXPORT int slim_attn_decode_split(const slim_cache_t *cache, const void *q, const int32_t *kv_len, int32_t B,
+                                       int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
+                                       size_t workspace_bytes, void *stream)
+{
+    bool launch;
+    int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (q == nullptr || kv_len == nullptr || ((uintptr_t)q & 15)) return SLIM_ERR_INVALID_ARG;
+    return launch_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_attn_decode_merge(const slim_cache_t *cache, void *out, const int32_t *kv_len, int32_t B,
+                                       int32_t max_kv, int32_t Hq, const void *workspace, size_t workspace_bytes,
+                                       void *stream)
+{
+    bool launch;
+    int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (out == nullptr || kv_len == nullptr || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
+    return launch_decode_merge(cache, out, kv_len, B, max_kv, Hq, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out, const int32_t *kv_len,
+                                 int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
+                                 size_t workspace_bytes, void *stream)
+{
+    bool launch;
+    int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (q == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
+    rc = launch_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+    if (rc != SLIM_OK) return rc;
+    return launch_decode_merge(cache, out, kv_len, B, max_kv, Hq, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv)
+{
+    if (B <= 0 || Hq <= 0 || Hkv <= 0) return 0;
+    return ((size_t)2 * B * Hq + (size_t)2 * B * Hkv) * SLIM_HEAD_DIM * 2;
+}
+
+SLIM_EXPORT int slim_decode_step_host(const slim_cache_t *cache, const void *q_host, const void *k_new_host,
+                                      const void *v_new_host, void *out_host, void *staging, size_t staging_bytes,
+                                      const int32_t *cu_new, const int32_t *start_pos, const int32_t *kv_len,
+                                      int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
+                                      size_t workspace_bytes, void *stream)
+{
+    bool launch;
+    int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (q_host == nullptr || k_new_host == nullptr || v_new_host == nullptr || out_host == nullptr ||
+        cu_new == nullptr || start_pos == nullptr || kv_len == nullptr)
+        return SLIM_ERR_INVALID_ARG;
+    const int Hkv = cache->num_kv_heads;
+    if (staging == nullptr || ((uintptr_t)staging & 15) || staging_bytes < slim_step_staging_bytes(B, Hq, Hkv))
+        return SLIM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t q_bytes = (size_t)B * Hq * SLIM_HEAD_DIM * 2, kv_bytes = (size_t)B * Hkv * SLIM_HEAD_DIM * 2;
+    char *d_q = static_cast<char *>(staging), *d_k = d_q + q_bytes, *d_v = d_k + kv_bytes, *d_o = d_v + kv_bytes;
+    SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, k_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, v_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    rc = launch_append(cache, d_k, d_v, cu_new, start_pos, B, 1, st);
+    if (rc != SLIM_OK) return rc;
+    rc = launch_decode_split(cache, d_q, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
+    if (rc != SLIM_OK) return rc;
+    rc = launch_decode_merge(cache, d_o, kv_len, B, max_kv, Hq, workspace, st);
+    if (rc != SLIM_OK) return rc;
+    SLIM_CUDA_TRY(cudaMemcpyAsync(out_host, d_o, q_bytes, cudaMemcpyDeviceToHost, st));
+    return SLIM_OK;
 }
 
 SLIM_EXPORT size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q,

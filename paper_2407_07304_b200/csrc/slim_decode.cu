@@ -307,12 +307,12 @@ static int launch_split(const DecodeParams &p, int B, cudaStream_t stream)
     return SLIM_OK;
 }
 
-int launch_decode(const slim_cache_t *c, const void *q, void *out, const int32_t *kv_len, int B, int max_kv,
-                  int Hq, float sm_scale, void *workspace, cudaStream_t stream)
+static DecodeParams make_params(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv,
+                                int Hq, float sm_scale, void *workspace, int &C)
 {
-    const int Hkv = c->num_kv_heads, G = Hq / Hkv;
+    const int Hkv = c->num_kv_heads;
     const int cp = decode_chunk_pages(B, Hkv, max_kv);
-    const int C = cp * kPageTokens;
+    C = cp * kPageTokens;
     DecodeParams p;
     p.codes = c->codes;
     p.scales = c->scales;
@@ -321,24 +321,33 @@ int launch_decode(const slim_cache_t *c, const void *q, void *out, const int32_t
     p.q = static_cast<const __nv_bfloat16 *>(q);
     p.Hq = Hq;
     p.Hkv = Hkv;
-    p.G = G;
+    p.G = Hq / Hkv;
     p.max_pages_per_seq = c->max_pages_per_seq;
     p.num_pages = c->num_pages;
     p.n_chunks = (max_kv + C - 1) / C;
     p.scale_log2e = sm_scale * kLog2e;
     p.part_o = static_cast<float *>(workspace);
     p.part_ml = p.part_o + (size_t)B * Hq * p.n_chunks * kHeadDim;
+    return p;
+}
 
-    if (p.n_chunks > 0) {
-        int rc;
-        if (G == 1)
-            rc = cp == 2 ? launch_split<1, 2>(p, B, stream) : launch_split<1, 1>(p, B, stream);
-        else if (G <= 8)
-            rc = cp == 2 ? launch_split<8, 2>(p, B, stream) : launch_split<8, 1>(p, B, stream);
-        else
-            rc = cp == 2 ? launch_split<16, 2>(p, B, stream) : launch_split<16, 1>(p, B, stream);
-        if (rc != SLIM_OK) return rc;
-    }
+int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv, int Hq,
+                        float sm_scale, void *workspace, cudaStream_t stream)
+{
+    int C;
+    const DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
+    if (p.n_chunks == 0) return SLIM_OK;
+    const int cp = C / kPageTokens;
+    if (p.G == 1) return cp == 2 ? launch_split<1, 2>(p, B, stream) : launch_split<1, 1>(p, B, stream);
+    if (p.G <= 8) return cp == 2 ? launch_split<8, 2>(p, B, stream) : launch_split<8, 1>(p, B, stream);
+    return cp == 2 ? launch_split<16, 2>(p, B, stream) : launch_split<16, 1>(p, B, stream);
+}
+
+int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
+                        const void *workspace, cudaStream_t stream)
+{
+    int C;
+    const DecodeParams p = make_params(c, nullptr, kv_len, B, max_kv, Hq, 1.f, const_cast<void *>(workspace), C);
     const int rows = B * Hq;
     slim_decode_merge_kernel<<<(rows + 3) / 4, 128, 0, stream>>>(p.part_o, p.part_ml, kv_len,
                                                                  static_cast<__nv_bfloat16 *>(out), B, Hq,
