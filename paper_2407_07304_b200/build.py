@@ -33,7 +33,7 @@ def build(force=False, verbose=False):
            "-shared", "-Xcompiler", "-fPIC", "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-lcuda"]
+    cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
     return LIB
 

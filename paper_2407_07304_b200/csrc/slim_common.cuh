@@ -154,12 +154,14 @@ struct QFrag {
 };
 
 // row_lo / row_hi: the 128 bf16 of A-row g and A-row g + 8 (nullptr = zero row).
+// With HI == false the upper eight rows are known to be zero and are not touched.
+template <bool HI = true>
 __device__ __forceinline__ void load_q_frag(QFrag &qf, const __nv_bfloat16 *row_lo, const __nv_bfloat16 *row_hi,
                                             int t, float &pow2_lo, float &pow2_hi)
 {
     float x[2][32];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
+    for (int r = 0; r < (HI ? 2 : 1); ++r) {
         const __nv_bfloat16 *row = r ? row_hi : row_lo;
         if (row != nullptr) {
             const uint4 *src = reinterpret_cast<const uint4 *>(row + 32 * t);
@@ -178,9 +180,9 @@ __device__ __forceinline__ void load_q_frag(QFrag &qf, const __nv_bfloat16 *row_
             for (int i = 0; i < 32; ++i) x[r][i] = 0.f;
         }
     }
-    float p2[2];
+    float p2[2] = {1.f, 1.f};
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
+    for (int r = 0; r < (HI ? 2 : 1); ++r) {
         float am = 0.f;
 #pragma unroll
         for (int i = 0; i < 32; ++i) am = fmaxf(am, fabsf(x[r][i]));
@@ -194,9 +196,9 @@ __device__ __forceinline__ void load_q_frag(QFrag &qf, const __nv_bfloat16 *row_
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         qf.a[j][0] = pack_half2(x[0][4 * j + 0], x[0][4 * j + 2]);
-        qf.a[j][1] = pack_half2(x[1][4 * j + 0], x[1][4 * j + 2]);
+        qf.a[j][1] = HI ? pack_half2(x[1][4 * j + 0], x[1][4 * j + 2]) : 0u;
         qf.a[j][2] = pack_half2(x[0][4 * j + 1], x[0][4 * j + 3]);
-        qf.a[j][3] = pack_half2(x[1][4 * j + 1], x[1][4 * j + 3]);
+        qf.a[j][3] = HI ? pack_half2(x[1][4 * j + 1], x[1][4 * j + 3]) : 0u;
     }
     pow2_lo = p2[0];
     pow2_hi = p2[1];

@@ -22,6 +22,9 @@
 namespace slim {
 
 constexpr int kDecodeThreads = 128;
+constexpr int kDecodeWarps = 4;
+constexpr int kWarpTok = 64;                              // tokens owned by one warp
+constexpr int kChunkTok = kDecodeWarps * kWarpTok;        // tokens per thread block (two pages)
 
 struct DecodeParams {
     const int8_t *codes;
@@ -36,207 +39,219 @@ struct DecodeParams {
     float scale_log2e;        // sm_scale * log2(e)
 };
 
-template <int ROWS, int CP>
-struct DecodeSmem {
-    static constexpr int C = CP * kPageTokens;          // tokens per chunk
-    static constexpr int PSTRIDE = C + 8;               // halfs; +16 bytes keeps A-fragment reads conflict-free
-    static constexpr size_t kOffK = 0;
-    static constexpr size_t kOffV = kOffK + (size_t)C * kHeadDim;
-    static constexpr size_t kOffKs = kOffV + (size_t)C * kHeadDim;
-    static constexpr size_t kOffVs = kOffKs + (size_t)C * 4;
-    static constexpr size_t kOffS = kOffVs + (size_t)C * 4;
-    static constexpr size_t kOffP = kOffS + (size_t)ROWS * C * 4;
-    static constexpr size_t kBytes = kOffP + (size_t)ROWS * PSTRIDE * 2;
+// Shared memory of one warp: its 64 tokens' K and V rows (swizzled, see swz_row_piece) and
+// scales.  After the warp has consumed them the same bytes hold its partial result.
+struct __align__(128) WarpBuf {
+    int8_t k[kWarpTok * kHeadDim];
+    int8_t v[kWarpTok * kHeadDim];
+    float ks[kWarpTok];
+    float vs[kWarpTok];
 };
+constexpr int kORowStride = 144;   // floats per partial-output row: four 32-float groups padded to 36
 
-// ROWS: query heads per kv head, rounded up to 1, 8 or 16.  CP: pages per chunk (1 or 2).
-template <int ROWS, int CP>
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ROWS: query heads per kv head, rounded up to 8 or 16 (rows of the 16-row MMA tile in use).
+//
+// A block owns 256 consecutive tokens of one (sequence, kv head); each of its four warps owns
+// 64 of them and works alone: it asks for its K rows, V rows and scales with 16-byte
+// asynchronous copies (all in flight at once), then follows the SlimAttention order on its
+// slice - all 64 scores, one softmax over them, then the product with V - entirely in
+// registers.  The four slices are merged through shared memory and written as one partial.
+template <int ROWS>
 __global__ void __launch_bounds__(kDecodeThreads)
 slim_decode_split_kernel(const DecodeParams p)
 {
-    using L = DecodeSmem<ROWS, CP>;
-    constexpr int C = L::C;
     extern __shared__ __align__(128) unsigned char smem[];
-    int8_t *kbuf = reinterpret_cast<int8_t *>(smem + L::kOffK);
-    int8_t *vbuf = reinterpret_cast<int8_t *>(smem + L::kOffV);
-    float *ksc = reinterpret_cast<float *>(smem + L::kOffKs);
-    float *vsc = reinterpret_cast<float *>(smem + L::kOffVs);
-    float *S = reinterpret_cast<float *>(smem + L::kOffS);
-    __half *P = reinterpret_cast<__half *>(smem + L::kOffP);
-
     const int chunk = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int len = min(p.kv_len[b], p.max_pages_per_seq * kPageTokens);
-    const int n_tok = min(C, len - chunk * C);   // valid tokens of this chunk
+    const int n_tok = min(kChunkTok, len - chunk * kChunkTok);   // valid tokens of this block
     if (n_tok <= 0) return;
+    WarpBuf &wb = reinterpret_cast<WarpBuf *>(smem)[warp];
+    const int n_w = max(0, min(kWarpTok, n_tok - warp * kWarpTok));   // valid tokens of this warp
+    const int h0 = head * p.G;
 
-    // ---- ask for the whole chunk: K pages (each with its page's K and V scales), then V pages
-    const int32_t *bt = p.block_table + (size_t)b * p.max_pages_per_seq + chunk * CP;
-    int page[CP];
+    float o[16][4];
 #pragma unroll
-    for (int pg = 0; pg < CP; ++pg) {
-        int id = (pg * kPageTokens < n_tok) ? bt[pg] : 0;
-        page[pg] = (id >= 0 && id < p.num_pages) ? id : 0;
-    }
+    for (int i = 0; i < 16; ++i)
 #pragma unroll
-    for (int kv = 0; kv < 2; ++kv) {
+        for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
+    float m_row[2] = {-INFINITY, -INFINITY}, l_row[2] = {0.f, 0.f};
+
+    if (n_w > 0) {
+        // ---- ask for everything this warp will read: K rows + both scale vectors, then V rows
+        int page = p.block_table[(size_t)b * p.max_pages_per_seq + chunk * 2 + (warp >> 1)];
+        page = (page >= 0 && page < p.num_pages) ? page : 0;
+        const int slot0 = (warp & 1) * kWarpTok;
+        {
+            const int r0 = lane >> 3, c = lane & 7;
+            // rows r0 + 4*it: (row & 7) alternates between r0 and r0 + 4
+            const uint32_t dsw[2] = {(uint32_t)((c ^ r0) << 4), (uint32_t)((c ^ (r0 + 4)) << 4)};
 #pragma unroll
-        for (int pg = 0; pg < CP; ++pg) {
-            const int rows = max(0, min(kPageTokens, n_tok - pg * kPageTokens));
-            const int8_t *src = p.codes + code_block_offset(page[pg], head, kv, p.Hkv);
-            const uint32_t dst = smem_u32((kv ? vbuf : kbuf) + pg * kPageTokens * kHeadDim);
-            for (int i = tid; i < rows * 8; i += kDecodeThreads) {
-                const int r = i >> 3, c = i & 7;
-                cp_async16(dst + swz_row_piece(r, c), src + r * kHeadDim + c * 16);
+            for (int kv = 0; kv < 2; ++kv) {
+                const int8_t *src = p.codes + code_block_offset(page, head, kv, p.Hkv) +
+                                    (size_t)(slot0 + r0) * kHeadDim + c * 16;
+                const uint32_t dst = smem_u32(kv ? wb.v : wb.k) + r0 * kHeadDim;
+#pragma unroll
+                for (int it = 0; it < 16; ++it)
+                    if (r0 + 4 * it < n_w) cp_async16(dst + it * 4 * kHeadDim + dsw[it & 1], src + it * 4 * kHeadDim);
+                if (kv == 0) {
+                    const int which = lane >> 4, qd = lane & 15;
+                    if (qd * 4 < n_w)
+                        cp_async16(smem_u32((which ? wb.vs : wb.ks) + qd * 4),
+                                   p.scales + scale_block_offset(page, head, which, p.Hkv) + slot0 + qd * 4);
+                }
+                cp_async_commit();
             }
-            if (kv == 0) {
-                const int quads = (rows + 3) >> 2;
-                for (int i = tid; i < 2 * quads; i += kDecodeThreads) {
-                    const int which = i >= quads;
-                    const int qd = which ? i - quads : i;
-                    const float *ssrc = p.scales + scale_block_offset(page[pg], head, which, p.Hkv) + qd * 4;
-                    cp_async16(smem_u32((which ? vsc : ksc) + pg * kPageTokens + qd * 4), ssrc);
+        }
+
+        // ---- query fragments (rows = the G heads of this kv head), while the copies fly
+        const __nv_bfloat16 *qbase = p.q + ((size_t)b * p.Hq + h0) * kHeadDim;
+        QFrag qf;
+        float pow2_lo, pow2_hi;
+        load_q_frag<(ROWS > 8)>(qf, (g < p.G) ? qbase + (size_t)g * kHeadDim : nullptr,
+                                (ROWS > 8 && g + 8 < p.G) ? qbase + (size_t)(g + 8) * kHeadDim : nullptr, t,
+                                pow2_lo, pow2_hi);
+        const float rs[2] = {pow2_lo * p.scale_log2e, pow2_hi * p.scale_log2e};
+
+        // ---- all scores of the slice (log2 units, V scale folded in): s[nt] = tokens 8nt + {2t, 2t+1}
+        cp_async_wait<1>();
+        __syncwarp();
+        float s[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s[nt][j] = 0.f;
+            if (nt * 8 < n_w) qk_tile(s[nt], qf, wb.k, nt * 8, g, t);
+        }
+        float rsv[8][2];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            const float2 sk = *reinterpret_cast<const float2 *>(wb.ks + nt * 8 + 2 * t);
+            const float2 sv = *reinterpret_cast<const float2 *>(wb.vs + nt * 8 + 2 * t);
+            const bool v0 = nt * 8 + 2 * t < n_w, v1 = nt * 8 + 2 * t + 1 < n_w;
+            const float l0 = log2_scale(sv.x), l1 = log2_scale(sv.y);
+            rsv[nt][0] = v0 ? recip_scale(sv.x) : 0.f;
+            rsv[nt][1] = v1 ? recip_scale(sv.y) : 0.f;
+            s[nt][0] = v0 ? fmaf(s[nt][0], sk.x * rs[0], l0) : -INFINITY;
+            s[nt][1] = v1 ? fmaf(s[nt][1], sk.y * rs[0], l1) : -INFINITY;
+            if (ROWS > 8) {
+                s[nt][2] = v0 ? fmaf(s[nt][2], sk.x * rs[1], l0) : -INFINITY;
+                s[nt][3] = v1 ? fmaf(s[nt][3], sk.y * rs[1], l1) : -INFINITY;
+            }
+            m_row[0] = fmaxf(m_row[0], fmaxf(s[nt][0], s[nt][1]));
+            if (ROWS > 8) m_row[1] = fmaxf(m_row[1], fmaxf(s[nt][2], s[nt][3]));
+        }
+        // ---- one softmax over the slice: P = 2^(s' - m') as fp16 A-fragments, l = sum P / scale_v
+        uint32_t pa[4][4];
+#pragma unroll
+        for (int r = 0; r < (ROWS > 8 ? 2 : 1); ++r) {
+            m_row[r] = fmaxf(m_row[r], __shfl_xor_sync(0xffffffffu, m_row[r], 1));
+            m_row[r] = fmaxf(m_row[r], __shfl_xor_sync(0xffffffffu, m_row[r], 2));
+        }
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            const float e0 = fast_exp2(s[nt][0] - m_row[0]), e1 = fast_exp2(s[nt][1] - m_row[0]);
+            l_row[0] = fmaf(e0, rsv[nt][0], fmaf(e1, rsv[nt][1], l_row[0]));
+            pa[nt >> 1][(nt & 1) * 2] = pack_half2(e0, e1);
+            if (ROWS > 8) {
+                const float e2 = fast_exp2(s[nt][2] - m_row[1]), e3 = fast_exp2(s[nt][3] - m_row[1]);
+                l_row[1] = fmaf(e2, rsv[nt][0], fmaf(e3, rsv[nt][1], l_row[1]));
+                pa[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(e2, e3);
+            } else {
+                pa[nt >> 1][(nt & 1) * 2 + 1] = 0u;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < (ROWS > 8 ? 2 : 1); ++r) {
+            l_row[r] += __shfl_xor_sync(0xffffffffu, l_row[r], 1);
+            l_row[r] += __shfl_xor_sync(0xffffffffu, l_row[r], 2);
+        }
+
+        // ---- O = P . V over the slice in steps of 16 tokens; thread (g, t) supplies head dims
+        //      16g + [0, 16) of token rows 16ks + {2t, 2t+1, 2t+8, 2t+9}
+        cp_async_wait<0>();
+        __syncwarp();
+        const uint32_t voff0 = (uint32_t)((2 * t) * kHeadDim + ((g ^ (2 * t)) << 4));
+        const uint32_t voff1 = (uint32_t)((2 * t + 1) * kHeadDim + ((g ^ (2 * t + 1)) << 4));
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            if (ks * 16 < n_w) {
+                // rows past the slice's last token hold stale bytes: any byte converts to a finite
+                // fp16 and its P entry is zero, so they add nothing
+                const int8_t *vb = wb.v + ks * 16 * kHeadDim;
+                const uint4 w0 = *reinterpret_cast<const uint4 *>(vb + voff0);
+                const uint4 w1 = *reinterpret_cast<const uint4 *>(vb + voff1);
+                const uint4 w2 = *reinterpret_cast<const uint4 *>(vb + voff0 + 8 * kHeadDim);
+                const uint4 w3 = *reinterpret_cast<const uint4 *>(vb + voff1 + 8 * kHeadDim);
+                const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
+                const uint32_t a2[4] = {w2.x, w2.y, w2.z, w2.w}, a3[4] = {w3.x, w3.y, w3.z, w3.w};
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const uint32_t x01 = __byte_perm(a0[q4], a1[q4], 0x5410), x23 = __byte_perm(a0[q4], a1[q4], 0x7632);
+                    const uint32_t y01 = __byte_perm(a2[q4], a3[q4], 0x5410), y23 = __byte_perm(a2[q4], a3[q4], 0x7632);
+                    mma_f16_16816(o[4 * q4 + 0], pa[ks], cvt_bytes02(x01), cvt_bytes02(y01));
+                    mma_f16_16816(o[4 * q4 + 1], pa[ks], cvt_bytes13(x01), cvt_bytes13(y01));
+                    mma_f16_16816(o[4 * q4 + 2], pa[ks], cvt_bytes02(x23), cvt_bytes02(y23));
+                    mma_f16_16816(o[4 * q4 + 3], pa[ks], cvt_bytes13(x23), cvt_bytes13(y23));
                 }
             }
-            cp_async_commit();
         }
     }
 
-    // ---- query fragments (rows = the G heads of this kv head), while the copies fly
-    const int h0 = head * p.G;
-    const __nv_bfloat16 *qbase = p.q + ((size_t)b * p.Hq + h0) * kHeadDim;
-    QFrag qf;
-    float pow2_lo, pow2_hi;
-    load_q_frag(qf, (g < p.G) ? qbase + (size_t)g * kHeadDim : nullptr,
-                (ROWS > 8 && g + 8 < p.G) ? qbase + (size_t)(g + 8) * kHeadDim : nullptr, t, pow2_lo, pow2_hi);
-    const float rs_lo = pow2_lo * p.scale_log2e, rs_hi = pow2_hi * p.scale_log2e;
-
-    // ---- scores of the whole chunk -> S (log2 units)
-    auto score_page = [&](int pg) {
-        const int rows = n_tok - pg * kPageTokens;
+    // ---- this warp's partial (m, l, O) into its own buffer; O row r, dim d at r*144 + (d/32)*36 + d%32
+    __syncwarp();
+    float *ow = reinterpret_cast<float *>(wb.k);   // spans k and v: 16 KB >= 16 * 144 * 4
+    float *mw = wb.ks, *lw = wb.vs;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int tok0 = pg * kPageTokens + (warp * 4 + i) * 8;
-            if (tok0 - pg * kPageTokens >= rows) break;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            qk_tile(acc, qf, kbuf, tok0, g, t);
-            const float2 sk = *reinterpret_cast<const float2 *>(ksc + tok0 + 2 * t);
-            const float2 sv = *reinterpret_cast<const float2 *>(vsc + tok0 + 2 * t);
-            const float lx = log2_scale(sv.x), ly = log2_scale(sv.y);
-            if (ROWS == 1) {
-                if (g == 0)
-                    *reinterpret_cast<float2 *>(S + tok0 + 2 * t) =
-                        make_float2(fmaf(acc[0], sk.x * rs_lo, lx), fmaf(acc[1], sk.y * rs_lo, ly));
-            } else {
-                *reinterpret_cast<float2 *>(S + g * C + tok0 + 2 * t) =
-                    make_float2(fmaf(acc[0], sk.x * rs_lo, lx), fmaf(acc[1], sk.y * rs_lo, ly));
-                if (ROWS > 8)
-                    *reinterpret_cast<float2 *>(S + (g + 8) * C + tok0 + 2 * t) =
-                        make_float2(fmaf(acc[2], sk.x * rs_hi, lx), fmaf(acc[3], sk.y * rs_hi, ly));
+    for (int r = 0; r < (ROWS > 8 ? 2 : 1); ++r) {
+        const int row = g + 8 * r;
+        if (row < p.G) {
+            float *dst = ow + row * kORowStride + t * 36;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                *reinterpret_cast<float4 *>(dst + 4 * i) =
+                    make_float4(o[4 * i][2 * r], o[4 * i + 1][2 * r], o[4 * i + 2][2 * r], o[4 * i + 3][2 * r]);
+                *reinterpret_cast<float4 *>(dst + 16 + 4 * i) =
+                    make_float4(o[4 * i][2 * r + 1], o[4 * i + 1][2 * r + 1], o[4 * i + 2][2 * r + 1], o[4 * i + 3][2 * r + 1]);
+            }
+            if (t == 0) {
+                mw[row] = m_row[r];
+                lw[row] = l_row[r];
             }
         }
-    };
-    if (CP == 1) {
-        cp_async_wait<1>();
-        __syncthreads();
-        score_page(0);
-    } else {
-        cp_async_wait<3>();
-        __syncthreads();
-        score_page(0);
-        cp_async_wait<2>();
-        __syncthreads();
-        if (n_tok > kPageTokens) score_page(1);
     }
     __syncthreads();
 
-    // ---- one softmax per row over the chunk: P = 2^(s' - m') in fp16, l = sum P / scale_v in fp32
-    const int n_pad = (n_tok + 15) & ~15;
-    for (int r = warp; r < ROWS; r += 4) {
-        if (r >= p.G) break;
-        float m = -INFINITY;
-        for (int i = lane; i < n_tok; i += 32) m = fmaxf(m, S[r * C + i]);
-        m = warp_max(m);
-        float l = 0.f;
-        for (int i = lane; i < n_pad; i += 32) {
-            float e = 0.f;
-            if (i < n_tok) {
-                e = exp2f(S[r * C + i] - m);
-                l = fmaf(e, recip_scale(vsc[i]), l);
-            }
-            P[r * L::PSTRIDE + i] = __float2half_rn(e);
-        }
-        l = warp_sum(l);
-        if (lane == 0) {
-            float *ml = p.part_ml + (((size_t)b * p.Hq + h0 + r) * p.n_chunks + chunk) * 2;
-            ml[0] = m;
-            ml[1] = l;
-        }
-    }
-
-    // ---- O = P . V: warp w owns head dims [32w, 32w+32); contraction over tokens in steps of 16
-    float o[4][4];
+    // ---- merge the four slices (log-sum-exp identity); thread d writes head dim d of every row
+    const WarpBuf *all = reinterpret_cast<const WarpBuf *>(smem);
+    const int dpos = (tid >> 5) * 36 + (tid & 31);
+    for (int row = 0; row < p.G; ++row) {
+        float mm[kDecodeWarps], M = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
-    const int piece = 2 * warp + (g >> 2);
-    const int inner = (g & 3) * 4;
-    auto pv_page = [&](int pg) {
-        const int rows = n_tok - pg * kPageTokens;
-#pragma unroll 2
-        for (int ks = 0; ks < 8; ++ks) {
-            if (ks * 16 >= rows) break;
-            const int tok0 = pg * kPageTokens + ks * 16;
-            uint32_t a[4] = {0u, 0u, 0u, 0u};
-            if (g < p.G) {
-                a[0] = *reinterpret_cast<const uint32_t *>(P + g * L::PSTRIDE + tok0 + 2 * t);
-                a[2] = *reinterpret_cast<const uint32_t *>(P + g * L::PSTRIDE + tok0 + 2 * t + 8);
-            }
-            if (ROWS > 8 && g + 8 < p.G) {
-                a[1] = *reinterpret_cast<const uint32_t *>(P + (g + 8) * L::PSTRIDE + tok0 + 2 * t);
-                a[3] = *reinterpret_cast<const uint32_t *>(P + (g + 8) * L::PSTRIDE + tok0 + 2 * t + 8);
-            }
-            uint32_t w[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = tok0 + 2 * t + (i & 1) + (i >> 1) * 8;
-                // rows past the chunk's last token hold stale bytes: any byte converts to a finite
-                // fp16 and its P entry is zero, so they add nothing
-                w[i] = *reinterpret_cast<const uint32_t *>(vbuf + swz_row_piece(row, piece) + inner);
-            }
-            const uint32_t x01 = __byte_perm(w[0], w[1], 0x5410), x23 = __byte_perm(w[0], w[1], 0x7632);
-            const uint32_t y01 = __byte_perm(w[2], w[3], 0x5410), y23 = __byte_perm(w[2], w[3], 0x7632);
-            mma_f16_16816(o[0], a, cvt_bytes02(x01), cvt_bytes02(y01));
-            mma_f16_16816(o[1], a, cvt_bytes13(x01), cvt_bytes13(y01));
-            mma_f16_16816(o[2], a, cvt_bytes02(x23), cvt_bytes02(y23));
-            mma_f16_16816(o[3], a, cvt_bytes13(x23), cvt_bytes13(y23));
+        for (int w = 0; w < kDecodeWarps; ++w) {
+            mm[w] = all[w].ks[row];
+            M = fmaxf(M, mm[w]);
         }
-    };
-    if (CP == 1) {
-        cp_async_wait<0>();
-        __syncthreads();
-        pv_page(0);
-    } else {
-        cp_async_wait<1>();
-        __syncthreads();
-        pv_page(0);
-        cp_async_wait<0>();
-        __syncthreads();
-        if (n_tok > kPageTokens) pv_page(1);
-    }
-
-    // ---- unnormalised partial output; thread (g, t) holds dims 32w + 8t + [0, 8) of rows g and g + 8
-    const int d0 = 32 * warp + 8 * t;
-    if (g < p.G) {
-        float *dst = p.part_o + (((size_t)b * p.Hq + h0 + g) * p.n_chunks + chunk) * kHeadDim + d0;
-        *reinterpret_cast<float4 *>(dst) = make_float4(o[0][0], o[1][0], o[2][0], o[3][0]);
-        *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[0][1], o[1][1], o[2][1], o[3][1]);
-    }
-    if (ROWS > 8 && g + 8 < p.G) {
-        float *dst = p.part_o + (((size_t)b * p.Hq + h0 + g + 8) * p.n_chunks + chunk) * kHeadDim + d0;
-        *reinterpret_cast<float4 *>(dst) = make_float4(o[0][2], o[1][2], o[2][2], o[3][2]);
-        *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[0][3], o[1][3], o[2][3], o[3][3]);
+        float acc = 0.f, l = 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecodeWarps; ++w) {
+            const float f = fast_exp2(mm[w] - M);   // 0 for an empty slice (m = -inf)
+            l = fmaf(all[w].vs[row], f, l);
+            acc = fmaf(reinterpret_cast<const float *>(all[w].k)[row * kORowStride + dpos], f, acc);
+        }
+        const size_t slot = ((size_t)b * p.Hq + h0 + row) * p.n_chunks + chunk;
+        p.part_o[slot * kHeadDim + tid] = acc;
+        if (tid == 0) {
+            p.part_ml[slot * 2] = M;
+            p.part_ml[slot * 2 + 1] = l;
+        }
     }
 }
 
@@ -280,29 +295,21 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
 }
 
 // ---------------------------------------------------------------- host side
-int decode_chunk_pages(int B, int Hkv, int max_kv)
-{
-    // Two pages per chunk halves the partial traffic; one page per chunk gives short
-    // problems enough blocks to fill 148 SMs several times over.
-    const long long blocks2 = (long long)B * Hkv * ((max_kv + 255) / 256);
-    return blocks2 >= 4LL * 148 ? 2 : 1;
-}
-
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv)
 {
-    const int cp = decode_chunk_pages(B, Hkv, max_kv);
-    const size_t nc = (size_t)(max_kv + cp * kPageTokens - 1) / (cp * kPageTokens);
+    (void)Hkv;
+    const size_t nc = (size_t)(max_kv + kChunkTok - 1) / kChunkTok;
     return (size_t)B * Hq * nc * (kHeadDim + 2) * sizeof(float);
 }
 
-template <int ROWS, int CP>
+template <int ROWS>
 static int launch_split(const DecodeParams &p, int B, cudaStream_t stream)
 {
-    using L = DecodeSmem<ROWS, CP>;
-    SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_split_kernel<ROWS, CP>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes));
+    constexpr int kBytes = kDecodeWarps * (int)sizeof(WarpBuf);
+    SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_split_kernel<ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kBytes));
     dim3 grid((unsigned)p.n_chunks, (unsigned)p.Hkv, (unsigned)B);
-    slim_decode_split_kernel<ROWS, CP><<<grid, kDecodeThreads, L::kBytes, stream>>>(p);
+    slim_decode_split_kernel<ROWS><<<grid, kDecodeThreads, kBytes, stream>>>(p);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }
@@ -311,8 +318,7 @@ static DecodeParams make_params(const slim_cache_t *c, const void *q, const int3
                                 int Hq, float sm_scale, void *workspace, int &C)
 {
     const int Hkv = c->num_kv_heads;
-    const int cp = decode_chunk_pages(B, Hkv, max_kv);
-    C = cp * kPageTokens;
+    C = kChunkTok;
     DecodeParams p;
     p.codes = c->codes;
     p.scales = c->scales;
@@ -337,10 +343,7 @@ int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_
     int C;
     const DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
     if (p.n_chunks == 0) return SLIM_OK;
-    const int cp = C / kPageTokens;
-    if (p.G == 1) return cp == 2 ? launch_split<1, 2>(p, B, stream) : launch_split<1, 1>(p, B, stream);
-    if (p.G <= 8) return cp == 2 ? launch_split<8, 2>(p, B, stream) : launch_split<8, 1>(p, B, stream);
-    return cp == 2 ? launch_split<16, 2>(p, B, stream) : launch_split<16, 1>(p, B, stream);
+    return p.G <= 8 ? launch_split<8>(p, B, stream) : launch_split<16>(p, B, stream);
 }
 
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
