@@ -2,21 +2,27 @@
 //
 // The next-token phase is a matrix-vector product bound by memory bandwidth
 // (Section 2.2, Eq. 1: every cached byte is read once per generated token), so
-// the kernel is organised around keeping the whole key range in flight:
-// a thread block owns one (sequence, kv head, chunk of keys), asks for its whole
-// chunk with 16-byte asynchronous copies at once, and consumes it as it lands.
-// Inside a chunk the order is SlimAttention's (Section 2.1): all scores of the
-// chunk first, one softmax over them, then the product with V - no running
-// rescale.  The G = Hq / Hkv query heads that share the kv head form the rows of
-// a 16-row tensor-core tile, so each cached byte is converted and used once for
-// all of them.
+// the kernel is organised around keeping the whole key range in flight and
+// spending as few instructions per cached byte as possible.
+//
+//  * A thread block owns 256 consecutive tokens of one (sequence, kv head); each
+//    of its four warps owns 64 of them and asks for its K rows, V rows and scales
+//    with 16-byte asynchronous copies, all in flight at once.
+//  * The INT8 codes go to the tensor cores as they are (integer MMA, m16n8k32):
+//    no per-element conversion.  The other operand is a 16-bit fixed-point copy
+//    of Q (and later of the softmax weights P) split into a high and a low byte,
+//    two integer MMAs per tile, recombined exactly as 256 * hi + lo in int32.
+//    The G = Hq / Hkv query heads that share the kv head are the rows of the
+//    16-row tile, so each cached byte is used once for all of them.
+//  * Inside the block the order is SlimAttention's (Section 2.1): all 256 scores
+//    first, one softmax over them, then the product with V - no running rescale.
 //
 // The V scale of key j is folded into the softmax weight: with
 //   s'_j = s_j + log2(scale_v[j]),  m' = max_j s'_j,  P_j = 2^(s'_j - m')
 // the output is  o = (sum_j P_j * v_code_j) / (sum_j P_j / scale_v[j]),
 // identical to softmax(s) . (v_code * scale_v) because the factor 2^(-m') cancels.
-// P_j <= 1 is normalised by the row's largest contribution, which is what makes
-// its fp16 copy for the tensor cores safe whatever the spread of the V scales.
+// P_j <= 1 is normalised by the block's largest contribution, which is what
+// makes its 16-bit fixed-point copy safe whatever the spread of the V scales.
 #include "slim_common.cuh"
 
 namespace slim {
@@ -25,6 +31,8 @@ constexpr int kDecodeThreads = 128;
 constexpr int kDecodeWarps = 4;
 constexpr int kWarpTok = 64;                              // tokens owned by one warp
 constexpr int kChunkTok = kDecodeWarps * kWarpTok;        // tokens per thread block (two pages)
+constexpr float kQFix = 16384.f;                          // Q fixed point: |q / pow2| < 2  ->  |v| < 32768
+constexpr float kPFix = 65535.f;                          // P fixed point: P in [0, 1]     ->  v in [0, 65535]
 
 struct DecodeParams {
     const int8_t *codes;
@@ -40,14 +48,22 @@ struct DecodeParams {
 };
 
 // Shared memory of one warp: its 64 tokens' K and V rows (swizzled, see swz_row_piece) and
-// scales.  After the warp has consumed them the same bytes hold its partial result.
+// scales.  After the warp has consumed them the K/V bytes hold its partial result.
 struct __align__(128) WarpBuf {
     int8_t k[kWarpTok * kHeadDim];
     int8_t v[kWarpTok * kHeadDim];
     float ks[kWarpTok];
-    float vs[kWarpTok];
+    float vs[kWarpTok];    // V scales, then log2 of them
+    float rsv[kWarpTok];   // 1 / V scale
+    float red[32];         // [0,16): slice row maxima, [16,32): slice row sums
 };
-constexpr int kORowStride = 144;   // floats per partial-output row: four 32-float groups padded to 36
+// A warp's partial output lives in its (consumed) K bytes as [row][128] int32 with the 16-byte
+// chunk index of dim d XOR-ed by (row ^ 2 * (d / 32)) & 7, which spreads the fragment stores
+// over the banks.
+__device__ __forceinline__ int opart_word(int row, int d)
+{
+    return row * kHeadDim + ((((d >> 2) ^ ((row ^ (2 * (d >> 5))) & 7))) << 2) + (d & 3);
+}
 
 __device__ __forceinline__ float fast_exp2(float x)
 {
@@ -55,34 +71,115 @@ __device__ __forceinline__ float fast_exp2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float fast_rcp(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// D(16x8, s32) += A(16x32, s8 or u8, row) * B(32x8, s8, col)
+template <bool A_UNSIGNED>
+__device__ __forceinline__ void mma_i8_16832(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1)
+{
+    if (A_UNSIGNED)
+        asm volatile(
+            "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+            : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Round-to-nearest-even integer of x in [0, 2^22) as the low bits of x + 2^23.
+__device__ __forceinline__ uint32_t fix_bits(float x, float scale)
+{
+    return __float_as_uint(fmaf(x, scale, 8388608.f));
+}
+
+// 16-bit fixed-point copy of the query rows as integer-MMA A fragments.
+// Thread (g, t) covers head dims [32t, 32t + 32) of rows g and g + 8; MMA step s (0..3)
+// contracts dims 32t + 8s + [0, 4) (first half of k) and 32t + 8s + [4, 8) (second half),
+// which is the order the K bytes arrive in (two 16-byte pieces per token and thread).
+template <bool HI_ROWS>
+struct QFix {
+    uint32_t hi[HI_ROWS ? 2 : 1][8];   // signed high bytes,   word j = dims 32t + 4j + [0, 4)
+    uint32_t lo[HI_ROWS ? 2 : 1][8];   // unsigned low bytes
+    float pow2[2];
+};
+
+template <bool HI_ROWS>
+__device__ __forceinline__ void load_q_fix(QFix<HI_ROWS> &qf, const __nv_bfloat16 *row_lo, const __nv_bfloat16 *row_hi,
+                                           int t)
+{
+    qf.pow2[0] = qf.pow2[1] = 1.f;
+#pragma unroll
+    for (int r = 0; r < (HI_ROWS ? 2 : 1); ++r) {
+        const __nv_bfloat16 *row = r ? row_hi : row_lo;
+        float x[32];
+        if (row != nullptr) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(row + 32 * t);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = __ldg(src + i);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    x[i * 8 + 2 * k] = bf16_bits_to_float(w[k] & 0xFFFFu);
+                    x[i * 8 + 2 * k + 1] = bf16_bits_to_float(w[k] >> 16);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) x[i] = 0.f;
+        }
+        float am = 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) am = fmaxf(am, fabsf(x[i]));
+        am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, 1));
+        am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, 2));
+        qf.pow2[r] = pow2_floor(am);
+        const float f = pow2_recip(qf.pow2[r]) * kQFix;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            // v = round(x * f) in (-32768, 32768): as int16 bits, hi = v >> 8 (signed), lo = v & 255
+            uint32_t b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) b[i] = __float_as_uint(fmaf(x[4 * j + i], f, 12582912.f));   // 1.5 * 2^23 + v
+            const uint32_t p01 = __byte_perm(b[0], b[1], 0x5140);   // [lo0, lo1, hi0, hi1]
+            const uint32_t p23 = __byte_perm(b[2], b[3], 0x5140);
+            qf.lo[r][j] = __byte_perm(p01, p23, 0x5410);
+            qf.hi[r][j] = __byte_perm(p01, p23, 0x7632);
+        }
+    }
+}
 
 // ROWS: query heads per kv head, rounded up to 8 or 16 (rows of the 16-row MMA tile in use).
-//
-// A block owns 256 consecutive tokens of one (sequence, kv head); each of its four warps owns
-// 64 of them and works alone: it asks for its K rows, V rows and scales with 16-byte
-// asynchronous copies (all in flight at once), then follows the SlimAttention order on its
-// slice - all 64 scores, one softmax over them, then the product with V - entirely in
-// registers.  The four slices are merged through shared memory and written as one partial.
 template <int ROWS>
 __global__ void __launch_bounds__(kDecodeThreads)
 slim_decode_split_kernel(const DecodeParams p)
 {
+    constexpr bool HI = ROWS > 8;
+    constexpr int NR = HI ? 2 : 1;
     extern __shared__ __align__(128) unsigned char smem[];
     const int chunk = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int len = min(p.kv_len[b], p.max_pages_per_seq * kPageTokens);
     const int n_tok = min(kChunkTok, len - chunk * kChunkTok);   // valid tokens of this block
     if (n_tok <= 0) return;
-    WarpBuf &wb = reinterpret_cast<WarpBuf *>(smem)[warp];
+    WarpBuf *all = reinterpret_cast<WarpBuf *>(smem);
+    WarpBuf &wb = all[warp];
     const int n_w = max(0, min(kWarpTok, n_tok - warp * kWarpTok));   // valid tokens of this warp
     const int h0 = head * p.G;
 
-    float o[16][4];
+    float s[8][2 * NR];           // scores of the slice: s[nt] = tokens 8nt + {2t, 2t+1} of rows g (and g + 8)
+    float m_loc[NR];
 #pragma unroll
-    for (int i = 0; i < 16; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) o[i][j] = 0.f;
-    float m_row[2] = {-INFINITY, -INFINITY}, l_row[2] = {0.f, 0.f};
+    for (int r = 0; r < NR; ++r) m_loc[r] = -INFINITY;
 
     if (n_w > 0) {
         // ---- ask for everything this warp will read: K rows + both scale vectors, then V rows
@@ -111,143 +208,214 @@ slim_decode_split_kernel(const DecodeParams p)
             }
         }
 
-        // ---- query fragments (rows = the G heads of this kv head), while the copies fly
+        // ---- fixed-point query fragments (rows = the G heads of this kv head), while the copies fly
         const __nv_bfloat16 *qbase = p.q + ((size_t)b * p.Hq + h0) * kHeadDim;
-        QFrag qf;
-        float pow2_lo, pow2_hi;
-        load_q_frag<(ROWS > 8)>(qf, (g < p.G) ? qbase + (size_t)g * kHeadDim : nullptr,
-                                (ROWS > 8 && g + 8 < p.G) ? qbase + (size_t)(g + 8) * kHeadDim : nullptr, t,
-                                pow2_lo, pow2_hi);
-        const float rs[2] = {pow2_lo * p.scale_log2e, pow2_hi * p.scale_log2e};
+        QFix<HI> qf;
+        load_q_fix<HI>(qf, (g < p.G) ? qbase + (size_t)g * kHeadDim : nullptr,
+                       (HI && g + 8 < p.G) ? qbase + (size_t)(g + 8) * kHeadDim : nullptr, t);
+        float rs[NR];
+#pragma unroll
+        for (int r = 0; r < NR; ++r) rs[r] = qf.pow2[r] * p.scale_log2e * (1.f / kQFix);
 
-        // ---- all scores of the slice (log2 units, V scale folded in): s[nt] = tokens 8nt + {2t, 2t+1}
         cp_async_wait<1>();
         __syncwarp();
-        float s[8][4];
+        // per-token log2 and reciprocal of the V scale, once per token (lane = token)
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) s[nt][j] = 0.f;
-            if (nt * 8 < n_w) qk_tile(s[nt], qf, wb.k, nt * 8, g, t);
-        }
-        float rsv[8][2];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            const float2 sk = *reinterpret_cast<const float2 *>(wb.ks + nt * 8 + 2 * t);
-            const float2 sv = *reinterpret_cast<const float2 *>(wb.vs + nt * 8 + 2 * t);
-            const bool v0 = nt * 8 + 2 * t < n_w, v1 = nt * 8 + 2 * t + 1 < n_w;
-            const float l0 = log2_scale(sv.x), l1 = log2_scale(sv.y);
-            rsv[nt][0] = v0 ? recip_scale(sv.x) : 0.f;
-            rsv[nt][1] = v1 ? recip_scale(sv.y) : 0.f;
-            s[nt][0] = v0 ? fmaf(s[nt][0], sk.x * rs[0], l0) : -INFINITY;
-            s[nt][1] = v1 ? fmaf(s[nt][1], sk.y * rs[0], l1) : -INFINITY;
-            if (ROWS > 8) {
-                s[nt][2] = v0 ? fmaf(s[nt][2], sk.x * rs[1], l0) : -INFINITY;
-                s[nt][3] = v1 ? fmaf(s[nt][3], sk.y * rs[1], l1) : -INFINITY;
-            }
-            m_row[0] = fmaxf(m_row[0], fmaxf(s[nt][0], s[nt][1]));
-            if (ROWS > 8) m_row[1] = fmaxf(m_row[1], fmaxf(s[nt][2], s[nt][3]));
-        }
-        // ---- one softmax over the slice: P = 2^(s' - m') as fp16 A-fragments, l = sum P / scale_v
-        uint32_t pa[4][4];
-#pragma unroll
-        for (int r = 0; r < (ROWS > 8 ? 2 : 1); ++r) {
-            m_row[r] = fmaxf(m_row[r], __shfl_xor_sync(0xffffffffu, m_row[r], 1));
-            m_row[r] = fmaxf(m_row[r], __shfl_xor_sync(0xffffffffu, m_row[r], 2));
-        }
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            const float e0 = fast_exp2(s[nt][0] - m_row[0]), e1 = fast_exp2(s[nt][1] - m_row[0]);
-            l_row[0] = fmaf(e0, rsv[nt][0], fmaf(e1, rsv[nt][1], l_row[0]));
-            pa[nt >> 1][(nt & 1) * 2] = pack_half2(e0, e1);
-            if (ROWS > 8) {
-                const float e2 = fast_exp2(s[nt][2] - m_row[1]), e3 = fast_exp2(s[nt][3] - m_row[1]);
-                l_row[1] = fmaf(e2, rsv[nt][0], fmaf(e3, rsv[nt][1], l_row[1]));
-                pa[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(e2, e3);
+        for (int i = 0; i < 2; ++i) {
+            const int tok = lane + 32 * i;
+            if (tok < n_w) {
+                const float sv = fmaxf(wb.vs[tok], kMinScale);
+                wb.vs[tok] = __log2f(sv);
+                wb.rsv[tok] = fast_rcp(sv);
             } else {
-                pa[nt >> 1][(nt & 1) * 2 + 1] = 0u;
+                wb.rsv[tok] = 0.f;
+            }
+        }
+        __syncwarp();
+
+        // ---- all scores of the slice: integer MMAs straight from the K bytes
+        const uint32_t koff0 = (uint32_t)(g * kHeadDim + (((2 * t) ^ g) << 4));
+        const uint32_t koff1 = (uint32_t)(g * kHeadDim + (((2 * t + 1) ^ g) << 4));
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            if (nt * 8 < n_w) {
+                const int8_t *kb = wb.k + nt * 8 * kHeadDim;
+                const uint4 lo4 = *reinterpret_cast<const uint4 *>(kb + koff0);
+                const uint4 hi4 = *reinterpret_cast<const uint4 *>(kb + koff1);
+                const uint32_t w[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+                int ah[4] = {0, 0, 0, 0}, al[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int st = 0; st < 4; ++st) {
+                    mma_i8_16832<false>(ah, qf.hi[0][2 * st], HI ? qf.hi[NR - 1][2 * st] : 0u, qf.hi[0][2 * st + 1],
+                                        HI ? qf.hi[NR - 1][2 * st + 1] : 0u, w[2 * st], w[2 * st + 1]);
+                    mma_i8_16832<true>(al, qf.lo[0][2 * st], HI ? qf.lo[NR - 1][2 * st] : 0u, qf.lo[0][2 * st + 1],
+                                       HI ? qf.lo[NR - 1][2 * st + 1] : 0u, w[2 * st], w[2 * st + 1]);
+                }
+                const float2 sk = *reinterpret_cast<const float2 *>(wb.ks + nt * 8 + 2 * t);
+                const float2 lv = *reinterpret_cast<const float2 *>(wb.vs + nt * 8 + 2 * t);
+                const bool v0 = nt * 8 + 2 * t < n_w, v1 = nt * 8 + 2 * t + 1 < n_w;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    const float x0 = (float)((ah[2 * r] << 8) + al[2 * r]);
+                    const float x1 = (float)((ah[2 * r + 1] << 8) + al[2 * r + 1]);
+                    s[nt][2 * r] = v0 ? fmaf(x0, sk.x * rs[r], lv.x) : -INFINITY;
+                    s[nt][2 * r + 1] = v1 ? fmaf(x1, sk.y * rs[r], lv.y) : -INFINITY;
+                    m_loc[r] = fmaxf(m_loc[r], fmaxf(s[nt][2 * r], s[nt][2 * r + 1]));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 2 * NR; ++j) s[nt][j] = -INFINITY;
             }
         }
 #pragma unroll
-        for (int r = 0; r < (ROWS > 8 ? 2 : 1); ++r) {
-            l_row[r] += __shfl_xor_sync(0xffffffffu, l_row[r], 1);
-            l_row[r] += __shfl_xor_sync(0xffffffffu, l_row[r], 2);
+        for (int r = 0; r < NR; ++r) {
+            m_loc[r] = fmaxf(m_loc[r], __shfl_xor_sync(0xffffffffu, m_loc[r], 1));
+            m_loc[r] = fmaxf(m_loc[r], __shfl_xor_sync(0xffffffffu, m_loc[r], 2));
+        }
+    }
+    // ---- block-wide row maxima
+    if (t == 0) {
+#pragma unroll
+        for (int r = 0; r < NR; ++r) wb.red[g + 8 * r] = m_loc[r];
+    }
+    __syncthreads();
+    float m_blk[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+        m_blk[r] = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kDecodeWarps; ++w) m_blk[r] = fmaxf(m_blk[r], all[w].red[g + 8 * r]);
+    }
+
+    float l_loc[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) l_loc[r] = 0.f;
+    int *ow = reinterpret_cast<int *>(wb.k);   // this warp's partial output: 16 rows x 128 int32 = the K bytes
+
+    if (n_w > 0) {
+        // ---- one softmax over the block's 256 scores: P = 2^(s' - m') in 16-bit fixed point, as
+        //      high-byte and low-byte A fragments of the two 32-token MMA steps; l = sum P / scale_v
+        uint32_t pa_hi[2][2 * NR], pa_lo[2][2 * NR];
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    // k slots 4t + {0,1,2,3} <- tokens of tiles (4ks + 2half, 4ks + 2half + 1), columns 2t, 2t+1
+                    uint32_t bits[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int nt = 4 * ks + 2 * half + (i >> 1);
+                        const float e = fast_exp2(s[nt][2 * r + (i & 1)] - m_blk[r]);
+                        l_loc[r] = fmaf(e, wb.rsv[nt * 8 + 2 * t + (i & 1)], l_loc[r]);
+                        bits[i] = fix_bits(e, kPFix);
+                    }
+                    const uint32_t p01 = __byte_perm(bits[0], bits[1], 0x5140);   // [lo0, lo1, hi0, hi1]
+                    const uint32_t p23 = __byte_perm(bits[2], bits[3], 0x5140);
+                    pa_lo[ks][NR * half + r] = __byte_perm(p01, p23, 0x5410);
+                    pa_hi[ks][NR * half + r] = __byte_perm(p01, p23, 0x7632);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+            l_loc[r] += __shfl_xor_sync(0xffffffffu, l_loc[r], 1);
+            l_loc[r] += __shfl_xor_sync(0xffffffffu, l_loc[r], 2);
         }
 
-        // ---- O = P . V over the slice in steps of 16 tokens; thread (g, t) supplies head dims
-        //      16g + [0, 16) of token rows 16ks + {2t, 2t+1, 2t+8, 2t+9}
+        // ---- O = P . V: integer MMAs over 32-token steps.  Thread (g, t) supplies head dims
+        //      16g + [0, 16) (one 16-byte piece per token row) of token rows
+        //      32ks + {2t, 2t+1, 8+2t, 9+2t} (first half of k) and + 16 (second half); the bytes of
+        //      four rows are transposed in registers into per-dim words.  Two passes of eight dims.
         cp_async_wait<0>();
         __syncwarp();
         const uint32_t voff0 = (uint32_t)((2 * t) * kHeadDim + ((g ^ (2 * t)) << 4));
         const uint32_t voff1 = (uint32_t)((2 * t + 1) * kHeadDim + ((g ^ (2 * t + 1)) << 4));
+        __syncwarp();
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-            if (ks * 16 < n_w) {
-                // rows past the slice's last token hold stale bytes: any byte converts to a finite
-                // fp16 and its P entry is zero, so they add nothing
-                const int8_t *vb = wb.v + ks * 16 * kHeadDim;
-                const uint4 w0 = *reinterpret_cast<const uint4 *>(vb + voff0);
-                const uint4 w1 = *reinterpret_cast<const uint4 *>(vb + voff1);
-                const uint4 w2 = *reinterpret_cast<const uint4 *>(vb + voff0 + 8 * kHeadDim);
-                const uint4 w3 = *reinterpret_cast<const uint4 *>(vb + voff1 + 8 * kHeadDim);
-                const uint32_t a0[4] = {w0.x, w0.y, w0.z, w0.w}, a1[4] = {w1.x, w1.y, w1.z, w1.w};
-                const uint32_t a2[4] = {w2.x, w2.y, w2.z, w2.w}, a3[4] = {w3.x, w3.y, w3.z, w3.w};
+        for (int dh = 0; dh < 2; ++dh) {
+            int oh[8][4], ol[8][4];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const uint32_t x01 = __byte_perm(a0[q4], a1[q4], 0x5410), x23 = __byte_perm(a0[q4], a1[q4], 0x7632);
-                    const uint32_t y01 = __byte_perm(a2[q4], a3[q4], 0x5410), y23 = __byte_perm(a2[q4], a3[q4], 0x7632);
-                    mma_f16_16816(o[4 * q4 + 0], pa[ks], cvt_bytes02(x01), cvt_bytes02(y01));
-                    mma_f16_16816(o[4 * q4 + 1], pa[ks], cvt_bytes13(x01), cvt_bytes13(y01));
-                    mma_f16_16816(o[4 * q4 + 2], pa[ks], cvt_bytes02(x23), cvt_bytes02(y23));
-                    mma_f16_16816(o[4 * q4 + 3], pa[ks], cvt_bytes13(x23), cvt_bytes13(y23));
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) oh[i][j] = ol[i][j] = 0;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                if (ks * 32 < n_w) {
+                    // rows past the slice's last token hold stale bytes; their P entries are zero
+                    const int8_t *vb = wb.v + ks * 32 * kHeadDim + dh * 8;
+                    uint2 rw[8];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        rw[2 * q] = *reinterpret_cast<const uint2 *>(vb + voff0 + q * 8 * kHeadDim);
+                        rw[2 * q + 1] = *reinterpret_cast<const uint2 *>(vb + voff1 + q * 8 * kHeadDim);
+                    }
+#pragma unroll
+                    for (int wd = 0; wd < 2; ++wd) {
+                        uint32_t bfrag[2][4];   // [k half][dim within the word]
+#pragma unroll
+                        for (int kh = 0; kh < 2; ++kh) {
+                            const uint32_t r0 = wd ? rw[4 * kh].y : rw[4 * kh].x, r1 = wd ? rw[4 * kh + 1].y : rw[4 * kh + 1].x;
+                            const uint32_t r2 = wd ? rw[4 * kh + 2].y : rw[4 * kh + 2].x, r3 = wd ? rw[4 * kh + 3].y : rw[4 * kh + 3].x;
+                            const uint32_t t0 = __byte_perm(r0, r1, 0x5140), t1 = __byte_perm(r2, r3, 0x5140);
+                            const uint32_t t2 = __byte_perm(r0, r1, 0x7362), t3 = __byte_perm(r2, r3, 0x7362);
+                            bfrag[kh][0] = __byte_perm(t0, t1, 0x5410);
+                            bfrag[kh][1] = __byte_perm(t0, t1, 0x7632);
+                            bfrag[kh][2] = __byte_perm(t2, t3, 0x5410);
+                            bfrag[kh][3] = __byte_perm(t2, t3, 0x7632);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            mma_i8_16832<true>(oh[4 * wd + i], pa_hi[ks][0], HI ? pa_hi[ks][NR - 1] : 0u, pa_hi[ks][NR],
+                                               HI ? pa_hi[ks][2 * NR - 1] : 0u, bfrag[0][i], bfrag[1][i]);
+                            mma_i8_16832<true>(ol[4 * wd + i], pa_lo[ks][0], HI ? pa_lo[ks][NR - 1] : 0u, pa_lo[ks][NR],
+                                               HI ? pa_lo[ks][2 * NR - 1] : 0u, bfrag[0][i], bfrag[1][i]);
+                        }
+                    }
+                }
+            }
+            // this pass's eight dims per column: dims 32t + 16c + 8dh + i for columns n = 2t + c
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+                const int row = g + 8 * r;
+                if (row < p.G) {
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        int v[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[i] = (oh[i][2 * r + c] << 8) + ol[i][2 * r + c];
+                        const int d = 32 * t + 16 * c + 8 * dh;
+                        *reinterpret_cast<int4 *>(ow + opart_word(row, d)) = make_int4(v[0], v[1], v[2], v[3]);
+                        *reinterpret_cast<int4 *>(ow + opart_word(row, d + 4)) = make_int4(v[4], v[5], v[6], v[7]);
+                    }
                 }
             }
         }
+    } else {
+        // an empty slice contributes zeros
+        for (int i = lane; i < ROWS * kHeadDim; i += 32) ow[i] = 0;
     }
-
-    // ---- this warp's partial (m, l, O) into its own buffer; O row r, dim d at r*144 + (d/32)*36 + d%32
-    __syncwarp();
-    float *ow = reinterpret_cast<float *>(wb.k);   // spans k and v: 16 KB >= 16 * 144 * 4
-    float *mw = wb.ks, *lw = wb.vs;
+    if (t == 0) {
 #pragma unroll
-    for (int r = 0; r < (ROWS > 8 ? 2 : 1); ++r) {
-        const int row = g + 8 * r;
-        if (row < p.G) {
-            float *dst = ow + row * kORowStride + t * 36;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                *reinterpret_cast<float4 *>(dst + 4 * i) =
-                    make_float4(o[4 * i][2 * r], o[4 * i + 1][2 * r], o[4 * i + 2][2 * r], o[4 * i + 3][2 * r]);
-                *reinterpret_cast<float4 *>(dst + 16 + 4 * i) =
-                    make_float4(o[4 * i][2 * r + 1], o[4 * i + 1][2 * r + 1], o[4 * i + 2][2 * r + 1], o[4 * i + 3][2 * r + 1]);
-            }
-            if (t == 0) {
-                mw[row] = m_row[r];
-                lw[row] = l_row[r];
-            }
-        }
+        for (int r = 0; r < NR; ++r) wb.red[16 + g + 8 * r] = l_loc[r];
     }
     __syncthreads();
 
-    // ---- merge the four slices (log-sum-exp identity); thread d writes head dim d of every row
-    const WarpBuf *all = reinterpret_cast<const WarpBuf *>(smem);
-    const int dpos = (tid >> 5) * 36 + (tid & 31);
+    // ---- sum the four slices (same maximum, so integer partial outputs add exactly);
+    //      thread d writes head dim d of every row
     for (int row = 0; row < p.G; ++row) {
-        float mm[kDecodeWarps], M = -INFINITY;
+        const int dpos = opart_word(row, tid) - row * kHeadDim;
+        int acc = 0;
+        float l = 0.f, M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kDecodeWarps; ++w) {
-            mm[w] = all[w].ks[row];
-            M = fmaxf(M, mm[w]);
-        }
-        float acc = 0.f, l = 0.f;
-#pragma unroll
-        for (int w = 0; w < kDecodeWarps; ++w) {
-            const float f = fast_exp2(mm[w] - M);   // 0 for an empty slice (m = -inf)
-            l = fmaf(all[w].vs[row], f, l);
-            acc = fmaf(reinterpret_cast<const float *>(all[w].k)[row * kORowStride + dpos], f, acc);
+            acc += reinterpret_cast<const int *>(all[w].k)[row * kHeadDim + dpos];
+            l += all[w].red[16 + row];
+            M = fmaxf(M, all[w].red[row]);
         }
         const size_t slot = ((size_t)b * p.Hq + h0 + row) * p.n_chunks + chunk;
-        p.part_o[slot * kHeadDim + tid] = acc;
+        p.part_o[slot * kHeadDim + tid] = (float)acc * (1.f / kPFix);
         if (tid == 0) {
             p.part_ml[slot * 2] = M;
             p.part_ml[slot * 2 + 1] = l;
