@@ -182,6 +182,43 @@ int slim_decode_step_host(const slim_cache_t *cache, const void *q_host, const v
                           void *workspace, size_t workspace_bytes, void *stream);
 size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
 
+/*
+ * Decode attention for callers that cannot allocate device memory.  (The paper
+ * has no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Some hosts of this library are not allowed to call cudaMalloc at the point
+ * where they run attention: code running while a CUDA graph is being captured,
+ * a plug-in inside a serving runtime whose memory pool is owned and fully
+ * reserved by someone else, or a real-time loop that must not take the
+ * allocator's locks.  slim_attn_decode needs a workspace for the split pass's
+ * partial results; this variant keeps those partials in a fixed array that is
+ * part of the library image, so the caller passes inputs and outputs only.
+ * It computes exactly what slim_attn_decode computes.
+ *
+ *  - The array is SLIM_STATIC_SCRATCH_BYTES (8 MiB) of device memory on every
+ *    GPU that loads the library, held until the process exits.
+ *  - A problem whose partials do not fit
+ *    (slim_workspace_bytes(SLIM_PHASE_DECODE, ...) > SLIM_STATIC_SCRATCH_BYTES)
+ *    is rejected with SLIM_ERR_WORKSPACE and nothing is launched; use
+ *    slim_attn_decode with your own workspace for those.
+ *  - No cudaMalloc/cudaFree and no allocating library routine is called.  The
+ *    first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress, with that device current); make that first call
+ *    before starting any stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last
+ *    call left in it.  Nothing in it has to start at zero: every slot a call
+ *    reads was written by that same call's split pass.  Two calls whose kernels
+ *    can overlap on the GPU (different streams, no ordering between them) race
+ *    on the array and give wrong results; keep calls on one stream or order
+ *    them with events.
+ *
+ * Arguments as for slim_attn_decode, minus the workspace.
+ */
+#define SLIM_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
+int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
+                            const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                            void *stream);
+
 /* Scratch bytes needed by a phase (SLIM_PHASE_*) for the given shape; 0 on invalid arguments. */
 size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q, int32_t max_kv);
 

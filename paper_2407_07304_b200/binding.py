@@ -25,7 +25,7 @@ PAGE_TOKENS = 128
 
 EXPORTS = (
     "slim_kv_append", "slim_attn_prefill", "slim_attn_decode", "slim_attn_decode_split",
-    "slim_attn_decode_merge", "slim_decode_step_host", "slim_step_staging_bytes", "slim_workspace_bytes",
+    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step_host", "slim_step_staging_bytes", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -78,6 +78,8 @@ def lib():
         L.slim_attn_decode_split.restype = ctypes.c_int
         L.slim_attn_decode_merge.argtypes = [CP, P, P, I, I, I, P, Z, P]
         L.slim_attn_decode_merge.restype = ctypes.c_int
+        L.slim_attn_decode_static.argtypes = [CP, P, P, P, I, I, I, F, P]
+        L.slim_attn_decode_static.restype = ctypes.c_int
         L.slim_decode_step_host.argtypes = [CP, P, P, P, P, P, Z, P, P, P, I, I, I, F, P, Z, P]
         L.slim_decode_step_host.restype = ctypes.c_int
         L.slim_step_staging_bytes.argtypes = [I, I, I]
@@ -176,6 +178,18 @@ def slim_attn_decode_merge(cache, out, kv_len, B, max_kv, Hq, workspace, stream=
     rc = lib().slim_attn_decode_merge(ctypes.byref(cache.struct), _ptr(out), _ptr(kv_len), B, max_kv, Hq,
                                       _ptr(workspace), _nbytes(workspace), _stream(stream))
     _check(rc, "slim_attn_decode_merge")
+
+
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+
+
+def slim_attn_decode_static(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, stream=None):
+    """slim_attn_decode without a workspace argument: partials go to the library's built-in
+    8 MiB device array, for callers that may not allocate.  Calls sharing a device must not
+    overlap on the GPU."""
+    rc = lib().slim_attn_decode_static(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(kv_len), B, max_kv, Hq,
+                                       sm_scale, _stream(stream))
+    _check(rc, "slim_attn_decode_static")
 
 
 def slim_decode_step_host(cache, q_host, k_new_host, v_new_host, out_host, staging, cu_new, start_pos, kv_len,

@@ -528,3 +528,62 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
 }
 
 }  // namespace slim
+
+// ---------------------------------------------------------------- decode without a caller-provided workspace
+//
+// Scratch for slim_attn_decode_static: the split pass's partial results live in this
+// file-scope device array instead of a buffer the caller allocates.  Every GPU that loads
+// the library carries these bytes until the process exits, so the size is kept modest.
+static __device__ __align__(256) unsigned char g_static_decode_scratch[SLIM_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices];      // device address of the array, per device ordinal
+bool g_static_scratch_ready[kMaxDevices];
+}  // namespace
+
+// In host code the array's name only stands for the symbol; the address a kernel can use has
+// to be asked for, once per device, while that device is current.
+static int static_scratch_address(void **ptr)
+{
+    int dev = -1;
+    SLIM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SLIM_ERR_UNSUPPORTED;
+    if (!g_static_scratch_ready[dev]) {
+        void *addr = nullptr;
+        SLIM_CUDA_TRY(cudaGetSymbolAddress(&addr, g_static_decode_scratch));
+        g_static_scratch_ptr[dev] = addr;
+        g_static_scratch_ready[dev] = true;
+    }
+    *ptr = g_static_scratch_ptr[dev];
+    return SLIM_OK;
+}
+
+extern "C" __attribute__((visibility("default")))
+int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out, const int32_t *kv_len, int32_t B,
+                            int32_t max_kv, int32_t Hq, float sm_scale, void *stream)
+{
+    using namespace slim;
+    if (cache == nullptr || cache->codes == nullptr || cache->scales == nullptr || cache->block_table == nullptr)
+        return SLIM_ERR_INVALID_ARG;
+    if (cache->num_pages <= 0 || cache->num_kv_heads <= 0 || cache->max_pages_per_seq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (cache->page_tokens != SLIM_PAGE_TOKENS || cache->head_dim != SLIM_HEAD_DIM) return SLIM_ERR_UNSUPPORTED;
+    if (((uintptr_t)cache->codes & 15) || ((uintptr_t)cache->scales & 15)) return SLIM_ERR_INVALID_ARG;
+    if (B < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (Hq % cache->num_kv_heads != 0 || Hq / cache->num_kv_heads > 16) return SLIM_ERR_UNSUPPORTED;
+    if (B == 0) return SLIM_OK;
+    if (B > 65535 || cache->num_kv_heads > 65535) return SLIM_ERR_UNSUPPORTED;
+    if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
+    if (q == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
+    // the problem must fit the built-in scratch: there is nothing to fall back to
+    if (decode_workspace_bytes(B, Hq, cache->num_kv_heads, max_kv) > (size_t)SLIM_STATIC_SCRATCH_BYTES)
+        return SLIM_ERR_WORKSPACE;
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != SLIM_OK) return rc;
+    rc = launch_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, scratch, (cudaStream_t)stream);
+    if (rc != SLIM_OK) return rc;
+    return launch_decode_merge(cache, out, kv_len, B, max_kv, Hq, scratch, (cudaStream_t)stream);
+}
+
