@@ -315,7 +315,7 @@ def run_ours(args, rank, world, local_rank):
 
 # dram bytes read + written by one slim_decode_split_kernel launch on this workload, from the ncu
 # capture summarised under profiles/ ; None until a capture of the current kernel exists.
-TRAFFIC_PER_LAUNCH = None
+TRAFFIC_PER_LAUNCH = 284.74e6
 
 
 def extra_numbers(slim, workloads, dev):
