@@ -217,4 +217,4 @@ def slim_version():
 def workspace(phase, B, Hq, Hkv, max_q, max_kv, device="cuda"):
     """A torch uint8 buffer of the size the phase needs (at least 16 bytes)."""
     n = max(16, slim_workspace_bytes(phase, B, Hq, Hkv, max_q, max_kv))
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    return torch.zeros(n, dtype=torch.uint8, device=device)

@@ -24,6 +24,7 @@
 // P_j <= 1 is normalised by the block's largest contribution, which is what
 // makes its 16-bit fixed-point copy safe whatever the spread of the V scales.
 #include "slim_common.cuh"
+#include "slim_decode_params.cuh"
 
 namespace slim {
 
@@ -33,19 +34,6 @@ constexpr int kWarpTok = 64;                              // tokens owned by one
 constexpr int kChunkTok = kDecodeWarps * kWarpTok;        // tokens per thread block (two pages)
 constexpr float kQFix = 16384.f;                          // Q fixed point: |q / pow2| < 2  ->  |v| < 32768
 constexpr float kPFix = 65535.f;                          // P fixed point: P in [0, 1]     ->  v in [0, 65535]
-
-struct DecodeParams {
-    const int8_t *codes;
-    const float *scales;
-    const int32_t *block_table;
-    const int32_t *kv_len;
-    const __nv_bfloat16 *q;   // [B][Hq][128]
-    float *part_o;            // [B][Hq][n_chunks][128] unnormalised partial outputs
-    float *part_ml;           // [B][Hq][n_chunks][2]   (max in log2 units, sum)
-    int Hq, Hkv, G;
-    int max_pages_per_seq, num_pages, n_chunks;
-    float scale_log2e;        // sm_scale * log2(e)
-};
 
 // Shared memory of one warp: its 64 tokens' K and V rows (swizzled, see swz_row_piece) and
 // scales.  After the warp has consumed them the K/V bytes hold its partial result.
@@ -467,7 +455,7 @@ size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv)
 {
     (void)Hkv;
     const size_t nc = (size_t)(max_kv + kChunkTok - 1) / kChunkTok;
-    return (size_t)B * Hq * nc * (kHeadDim + 2) * sizeof(float);
+    return kDecodeStatusBytes + (size_t)B * Hq * nc * (kHeadDim + 2) * sizeof(float);
 }
 
 template <int ROWS>
@@ -500,7 +488,8 @@ static DecodeParams make_params(const slim_cache_t *c, const void *q, const int3
     p.num_pages = c->num_pages;
     p.n_chunks = (max_kv + C - 1) / C;
     p.scale_log2e = sm_scale * kLog2e;
-    p.part_o = static_cast<float *>(workspace);
+    p.status = static_cast<int *>(workspace);
+    p.part_o = reinterpret_cast<float *>(static_cast<char *>(workspace) + kDecodeStatusBytes);
     p.part_ml = p.part_o + (size_t)B * Hq * p.n_chunks * kHeadDim;
     return p;
 }
@@ -511,7 +500,7 @@ int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_
     int C;
     const DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
     if (p.n_chunks == 0) return SLIM_OK;
-    return p.G <= 8 ? launch_split<8>(p, B, stream) : launch_split<16>(p, B, stream);
+    return launch_decode_split_tc(p, B, stream);
 }
 
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,

@@ -1,0 +1,25 @@
+// Parameters shared by the decode split kernels and the merge kernel.
+#pragma once
+#include "slim_common.cuh"
+
+namespace slim {
+
+struct DecodeParams {
+    const int8_t *codes;
+    const float *scales;
+    const int32_t *block_table;
+    const int32_t *kv_len;
+    const __nv_bfloat16 *q;   // [B][Hq][128]
+    int *status;              // first word of the workspace: set to a SLIM_ERR_* code by a kernel whose wait ran out
+    float *part_o;            // [B][Hq][n_chunks][128] unnormalised partial outputs
+    float *part_ml;           // [B][Hq][n_chunks][2]   (max in log2 units, sum)
+    int Hq, Hkv, G;
+    int max_pages_per_seq, num_pages, n_chunks;
+    float scale_log2e;        // sm_scale * log2(e)
+};
+
+constexpr size_t kDecodeStatusBytes = 16;   // status word + padding in front of the partials
+
+int launch_decode_split_tc(const DecodeParams &p, int B, cudaStream_t stream);
+
+}  // namespace slim
