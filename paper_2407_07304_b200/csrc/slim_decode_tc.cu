@@ -61,7 +61,11 @@ slim_decode_split_tc_kernel(const DecodeParams p)
     extern __shared__ __align__(1024) unsigned char smem[];
     const int chunk = blockIdx.x, head = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int len = min(p.kv_len[b], p.max_pages_per_seq * kPageTokens);
+    // the page ids do not depend on the length: ask for both at once (two dependent round trips otherwise)
+    const int32_t *bt = p.block_table + (size_t)b * p.max_pages_per_seq + chunk * 2;
+    const int id0 = (chunk * 2 < p.max_pages_per_seq) ? __ldg(bt) : 0;
+    const int id1 = (chunk * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
+    const int len = min(__ldg(p.kv_len + b), p.max_pages_per_seq * kPageTokens);
     const int n_tok = min(kTcChunkTok, len - chunk * kTcChunkTok);   // valid tokens of this block
     if (n_tok <= 0) return;
     const int n_tiles = n_tok > kTileTok ? 2 : 1;
@@ -78,13 +82,9 @@ slim_decode_split_tc_kernel(const DecodeParams p)
 
     // ---- ask for the whole block: K tile 0 + its scales | K tile 1 + scales | V tile 0 | V tile 1
     {
-        const int32_t *bt = p.block_table + (size_t)b * p.max_pages_per_seq + chunk * 2;
-        int page[2];
+        int page[2] = {id0, id1};
 #pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int id = (t < n_tiles) ? bt[t] : 0;
-            page[t] = (id >= 0 && id < p.num_pages) ? id : 0;
-        }
+        for (int t = 0; t < 2; ++t) page[t] = (page[t] >= 0 && page[t] < p.num_pages) ? page[t] : 0;
         const int r0 = tid >> 3, c = tid & 7;
         const uint32_t dsw = (uint32_t)(r0 * kHeadDim + ((c ^ (r0 & 7)) << 4));   // rows r0 + 16 * it keep (row & 7)
 #pragma unroll
