@@ -374,11 +374,18 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-extra", action="store_true", help="skip the prefill context numbers")
+    ap.add_argument("--extra-only", action="store_true",
+                    help="run only the workload-3 prefill/append timings (for profiling that kernel) and print them")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.extra_only:
+        import torch
+        from paper_2407_07304_b200 import binding as slim, workloads
+        torch.cuda.set_device(local_rank)
+        print(json.dumps({"extra": extra_numbers(slim, workloads, torch.device("cuda", local_rank))}), flush=True)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)

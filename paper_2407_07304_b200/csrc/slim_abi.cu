@@ -1,4 +1,6 @@
 // C ABI of the library (declared in include/slim.h): argument validation and dispatch.
+#include <stdlib.h>
+
 #include "slim_common.cuh"
 
 #define SLIM_EXPORT extern "C" __attribute__((visibility("default")))
@@ -20,6 +22,9 @@ int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
                         const void *workspace, cudaStream_t stream);
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
+int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
+                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
+size_t prefill_workspace_bytes();
 int launch_prefill_mma(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                        int B, int max_q, int Hq, float sm_scale, cudaStream_t stream);
 
@@ -66,7 +71,13 @@ SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void
     if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
     const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
-    return launch_prefill_mma(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, (cudaStream_t)stream);
+    // SLIM_PREFILL_IMPL=mma selects the warp-level MMA kernel (kept for cross-checks); default is tcgen05
+    static const bool use_mma = [] {
+        const char *e = getenv("SLIM_PREFILL_IMPL");
+        return e != nullptr && e[0] == 'm';
+    }();
+    if (use_mma) return launch_prefill_mma(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, (cudaStream_t)stream);
+    return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream);
 }
 
 // Shared validation of the decode entry points; *launch is false for a valid no-op.
@@ -166,6 +177,7 @@ SLIM_EXPORT size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, in
 {
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || max_kv < 0 || max_q < 0) return 0;
     if (phase == SLIM_PHASE_DECODE) return decode_workspace_bytes(B, Hq, Hkv, max_kv);
+    if (phase == SLIM_PHASE_PREFILL) return prefill_workspace_bytes();
     return 0;
 }
 
