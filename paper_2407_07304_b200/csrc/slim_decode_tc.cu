@@ -180,6 +180,7 @@ slim_decode_split_tc_kernel(const DecodeParams p)
     }
 
     ok = tc::mbar_wait(bar_qk, 0);
+    __syncwarp();   // reconverge after the wait loop: the tensor-memory load below is warp-aligned
     tc::fence_after_sync();
 
     // ---- S^T from tensor memory: row = token, columns [hi | lo] per head
@@ -266,6 +267,7 @@ slim_decode_split_tc_kernel(const DecodeParams p)
         tc::commit(bar_pv);
     }
     ok = tc::mbar_wait(bar_pv, 0) && ok;
+    __syncwarp();
     tc::fence_after_sync();
 
     // ---- O^T from tensor memory: row = head dim, columns [hi | lo] per head; one partial per head

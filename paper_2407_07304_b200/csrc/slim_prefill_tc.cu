@@ -175,6 +175,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         for (int j = 0; j < T; ++j) {
             const int buf = j & 1;
             wait(bar(ptl::S_FULL, buf), (j >> 1) & 1);
+            __syncwarp();   // the wait loop may leave the lanes diverged; the tensor-memory ops below are warp-aligned
             tc::fence_after_sync();
             float s[128];
 #pragma unroll
@@ -206,6 +207,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
                 const float alpha = grow ? fast_exp2f(m_run - mt) : 1.f;   // m_run = -inf gives 0
                 wait(bar(ptl::SP_EMPTY, (j - 1) & 1), ((j - 1) >> 1) & 1);  // P.V of the previous tile is complete
+                __syncwarp();
                 tc::fence_after_sync();
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
@@ -244,6 +246,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
         if (T > 0) {
             wait(bar(ptl::SP_EMPTY, (T - 1) & 1), ((T - 1) >> 1) & 1);
+            __syncwarp();
             tc::fence_after_sync();
         }
         uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim);
