@@ -23,6 +23,8 @@
 // identical to softmax(s) . (v_code * scale_v) because the factor 2^(-m') cancels.
 // P_j <= 1 is normalised by the block's largest contribution, which is what
 // makes its 16-bit fixed-point copy safe whatever the spread of the V scales.
+#include <stdlib.h>
+
 #include "slim_common.cuh"
 #include "slim_decode_params.cuh"
 
@@ -500,7 +502,13 @@ int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_
     int C;
     const DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
     if (p.n_chunks == 0) return SLIM_OK;
-    return launch_decode_split_tc(p, B, stream);
+    // SLIM_DECODE_IMPL=oneshot selects the one-block-per-chunk kernel (kept for cross-checks)
+    static const bool oneshot = [] {
+        const char *e = getenv("SLIM_DECODE_IMPL");
+        return e != nullptr && e[0] == 'o';
+    }();
+    if (oneshot) return launch_decode_split_tc(p, B, stream);
+    return launch_decode_split_stream(c, p, B, stream);
 }
 
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,

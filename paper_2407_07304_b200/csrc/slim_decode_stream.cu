@@ -1,0 +1,504 @@
+// Decode split pass as a persistent streaming kernel (sm_100a): TMA ring -> tcgen05 -> partials.
+//
+// The next-token phase is bound by memory bandwidth (Section 2.2, Eq. 1: every cached byte is read once
+// per generated token).  The kernel therefore keeps the copy engine busy all the time and spends almost
+// no instructions per cached byte:
+//
+//  * One thread block per SM.  The work - every 256-token chunk of every (sequence, kv head) - is cut
+//    into one contiguous range per block.  A chunk is the unit of a partial result (m, l, O[128]).
+//  * Warp 8 is the producer: one thread walks the block's chunks and asks the TMA engine for each
+//    chunk's INT8 K tiles, V tiles, scales and query rows into a ring of three shared-memory slots
+//    (128-byte swizzled tiles, completion counted on mbarriers).  A ragged last tile is fetched in
+//    16-row boxes so that no byte beyond the chunk's tokens (rounded up to 16) is read.
+//  * Warps 0-3 and 4-7 are two consumer groups that take chunks alternately.  For its chunk a group
+//      - builds the query operand: a 14-bit fixed-point copy of the G = Hq/Hkv query rows of the kv
+//        head, two signed bytes per value (columns [high bytes | low bytes]);
+//      - S^T[token][head] = K_codes . Q^T by tcgen05.mma kind::i8: the INT8 codes are the operand as
+//        they are (the hybrid-dtype step of Section 2.2 happens inside the tensor core);
+//      - one softmax over the chunk's 256 scores per head (Section 2.1 order: all scores, softmax,
+//        then .V), thread = token, after a tensor-memory load;
+//      - O^T[dim][head] = V_codes^T . P^T, again kind::i8, V read MN-major straight from its
+//        token-major rows, P as 16-bit fixed point in two unsigned bytes;
+//      - recombines 256 * high + low exactly in int32 and writes the partial.
+//    While one group computes, the other group's chunk and the next chunk are in flight.
+//
+// The V scale is folded into the softmax weight (s'_j = s_j + log2 sv_j, P_j = 2^(s'_j - max s'),
+// o = sum P_j c_j / sum P_j / sv_j), so P <= 1 is normalised by the chunk's largest contribution.
+// Every wait is bounded; a wait that runs out raises the status word and the block drains and exits.
+#include <cuda.h>
+
+#include "slim_common.cuh"
+#include "slim_decode_params.cuh"
+#include "slim_tcgen05.cuh"
+#include "slim_tmap.cuh"
+
+namespace slim {
+
+constexpr int kStGroups = 2;
+constexpr int kStGroupThreads = 128;
+constexpr int kStThreads = kStGroups * kStGroupThreads + 32;   // two consumer groups + the producer warp
+constexpr int kStSlots = 3;
+constexpr int kStTile = 128;                                    // tokens per MMA tile (= one page)
+constexpr int kStChunk = 2 * kStTile;                           // tokens per chunk / partial
+constexpr int kStTailBox = 16;                                  // rows per TMA box of a ragged tile
+constexpr float kStQFix = 8192.f;      // |q / pow2| < 2  ->  |v| < 16384, high byte in [-64, 64]
+constexpr float kStPFix = 65535.f;
+constexpr uint32_t kStTmemCols = 256;  // 128 per group: S of two tiles + O
+
+static_assert(kStChunk == 256, "partials are indexed by 256-token chunks (decode_workspace_bytes, merge kernel)");
+
+template <int NH>
+struct StSmem {
+    static constexpr int N = 2 * NH;                        // MMA columns: [hi bytes of NH heads | lo bytes]
+    // one ring slot = one chunk
+    static constexpr uint32_t kK = 0;                       // two K tiles, 16 KB each
+    static constexpr uint32_t kV = 32768;                   // two V tiles
+    static constexpr uint32_t kKs = 65536;                  // 256 K scales
+    static constexpr uint32_t kVs = kKs + 1024;             // 256 V scales
+    static constexpr uint32_t kQraw = kVs + 1024;           // the kv head's query rows, bf16 [G][128]
+    static constexpr uint32_t kMeta = kQraw + NH * 256;     // int4: sequence, kv head, chunk, valid tokens
+    static constexpr uint32_t kSlotBytes = (kMeta + 16 + 1023) / 1024 * 1024;
+    static constexpr uint32_t kPTileBytes = N * 128;        // a P^T tile (aliases K tile 0 once the scores are out)
+    // per consumer group
+    static constexpr uint32_t kGroup0 = kStSlots * kSlotBytes;
+    static constexpr uint32_t kQop = 0;                     // query operand: N rows x 128 bytes, core-matrix layout
+    static constexpr uint32_t kRed = N * 128;               // floats: [NH][4] warp maxima, [NH][4] warp sums, [NH] row scales
+    static constexpr uint32_t kGroupBytes = (kRed + 9 * NH * 4 + 127) / 128 * 128;
+    // block-wide
+    static constexpr uint32_t kBar = kGroup0 + kStGroups * kGroupBytes;   // 13 mbarriers
+    static constexpr uint32_t kTmemSlot = kBar + 13 * 8;
+    static constexpr uint32_t kRange = kTmemSlot + 8;       // int[4]: chunks of this block, first sequence / head / chunk
+    static constexpr uint32_t kFail = kRange + 16;
+    static constexpr uint32_t kBytes = kFail + 8;
+    static_assert(2 * kPTileBytes <= 16384, "both P^T tiles live in K tile 0");
+    static_assert(kBytes <= 232448, "shared memory budget of one block");
+};
+
+// Byte offset of element (row n, k byte kb) of a K-major operand stored as 8x16-byte core matrices:
+// 16 bytes of k contiguous, 8 rows 16 bytes apart, next 16 k-bytes +128, next 8 rows +1024.
+__device__ __forceinline__ uint32_t st_core_off(int n, int kb)
+{
+    return (uint32_t)((n >> 3) * 1024 + (kb >> 4) * 128 + (n & 7) * 16 + (kb & 15));
+}
+
+// A sequence's cached tokens, never beyond the page table or the launch's max_kv.
+__device__ __forceinline__ int st_clamped_len(const DecodeParams &p, int b)
+{
+    const int cap = min(p.max_pages_per_seq * kPageTokens, p.n_chunks * kStChunk);
+    return min(max(__ldg(p.kv_len + b), 0), cap);
+}
+
+template <int NH>
+__global__ void __launch_bounds__(kStThreads, 1)
+slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __grid_constant__ CUtensorMap map_tail,
+                          const DecodeParams p, const int B)
+{
+    using L = StSmem<NH>;
+    constexpr int N = L::N;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::kBar;
+    auto bar_full_k = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto bar_full_v = [&](int s) { return bar0 + 8u * (uint32_t)(3 + s); };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (uint32_t)(6 + s); };
+    auto bar_mma_s = [&](int g) { return bar0 + 8u * (uint32_t)(9 + g); };
+    auto bar_mma_pv = [&](int g) { return bar0 + 8u * (uint32_t)(11 + g); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kTmemSlot);
+    int *range = reinterpret_cast<int *>(smem + L::kRange);
+    volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
+
+    if (tid == 0) {
+        for (int i = 0; i < 13; ++i) tc::mbar_init(bar0 + 8u * i, 1);
+        tc::mbar_init_fence();
+        *fail = 0;
+    }
+    if (warp == 8) {
+        tc::tmem_alloc(smem_u32(tmem_slot), kStTmemCols);
+        // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order
+        long long chunks_all = 0;
+        for (int base = 0; base < B; base += 32) {
+            const int b = base + lane;
+            const int nc = (b < B) ? (st_clamped_len(p, b) + kStChunk - 1) / kStChunk : 0;
+            chunks_all += __reduce_add_sync(0xffffffffu, nc);
+        }
+        const long long total = chunks_all * p.Hkv;
+        const long long i0 = total * blockIdx.x / gridDim.x, i1 = total * (blockIdx.x + 1) / gridDim.x;
+        int b0 = 0, head0 = 0, chunk0 = 0;
+        if (i1 > i0) {
+            long long prefix = 0;   // chunks of the sequences before `base`
+            for (int base = 0; base < B; base += 32) {
+                const int b = base + lane;
+                const int nc = (b < B) ? (st_clamped_len(p, b) + kStChunk - 1) / kStChunk : 0;
+                int incl = nc;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, (prefix + incl) * p.Hkv > i0);
+                if (hit != 0u) {
+                    const int l = __ffs(hit) - 1;
+                    const int nc_l = __shfl_sync(0xffffffffu, nc, l);
+                    const long long before = prefix + __shfl_sync(0xffffffffu, incl, l) - nc_l;
+                    const long long r = i0 - before * p.Hkv;   // < Hkv * nc_l
+                    b0 = base + l;
+                    head0 = (int)(r / nc_l);
+                    chunk0 = (int)(r % nc_l);
+                    break;
+                }
+                prefix += __shfl_sync(0xffffffffu, incl, 31);
+            }
+        }
+        if (lane == 0) {
+            range[0] = (int)(i1 - i0);
+            range[1] = b0;
+            range[2] = head0;
+            range[3] = chunk0;
+        }
+    } else {
+        // rows of the query operand that belong to no head stay zero for the whole launch
+        const int g = warp >> 2, gtid = tid & 127;
+        unsigned char *qop = smem + L::kGroup0 + g * L::kGroupBytes + L::kQop;
+        for (int i = gtid * 16; i < N * 128; i += kStGroupThreads * 16) *reinterpret_cast<uint4 *>(qop + i) = make_uint4(0, 0, 0, 0);
+    }
+    tc::fence_proxy_async();
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    const int cnt = range[0];
+    bool ok = true;
+    auto wait = [&](uint32_t mbar, uint32_t parity) {
+        if (!tc::mbar_wait(mbar, parity, (ok && *fail == 0) ? (1u << 18) : 1u)) {
+            ok = false;
+            *fail = 1;
+        }
+    };
+
+    if (warp == 8) {
+        // =========================================================== producer (one thread)
+        if (lane == 0 && cnt > 0) {
+            int b = range[1], head = range[2], chunk = range[3];
+            int len = st_clamped_len(p, b);
+            int nc = (len + kStChunk - 1) / kStChunk;
+            auto page_ids = [&](int bb, int cc) {
+                const int32_t *bt = p.block_table + (size_t)bb * p.max_pages_per_seq + cc * 2;
+                int2 r;
+                r.x = (cc * 2 < p.max_pages_per_seq) ? __ldg(bt) : 0;
+                r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
+                return r;
+            };
+            int2 pg = page_ids(b, chunk);
+            for (int n = 0; n < cnt; ++n) {
+                const int slot = n % kStSlots;
+                const uint32_t ph = (uint32_t)(n / kStSlots) & 1u;
+                const int cb = b, chead = head, cchunk = chunk;
+                const int n_tok = min(kStChunk, len - chunk * kStChunk);
+                const int2 cpg = pg;
+                // ---- the next chunk's coordinates and page ids, requested before this chunk's copies are issued
+                if (n + 1 < cnt) {
+                    if (++chunk == nc) {
+                        chunk = 0;
+                        if (++head == p.Hkv) {
+                            head = 0;
+                            do {
+                                ++b;
+                                len = (b < B) ? st_clamped_len(p, b) : kStChunk;   // b < B always holds inside the range
+                                nc = (len + kStChunk - 1) / kStChunk;
+                            } while (nc == 0);
+                        }
+                    }
+                    pg = page_ids(min(b, B - 1), chunk);
+                }
+                wait(bar_empty(slot), ph ^ 1u);
+                const uint32_t sl = sbase + slot * L::kSlotBytes;
+                *reinterpret_cast<int4 *>(smem + slot * L::kSlotBytes + L::kMeta) = make_int4(cb, chead, cchunk, n_tok);
+                int page[2] = {cpg.x, cpg.y};
+                int rows16[2];
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    page[t] = (page[t] >= 0 && page[t] < p.num_pages) ? page[t] : 0;
+                    const int rows = max(0, min(kStTile, n_tok - t * kStTile));
+                    rows16[t] = (rows + kStTailBox - 1) / kStTailBox * kStTailBox;
+                }
+                const uint32_t code_bytes = (uint32_t)(rows16[0] + rows16[1]) * kHeadDim;
+                const uint32_t q_bytes = (uint32_t)p.G * kHeadDim * 2u;
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+                    const uint32_t full = kv ? bar_full_v(slot) : bar_full_k(slot);
+                    // K barrier: K tiles + both scale vectors + the query rows; V barrier: V tiles
+                    tc::mbar_arrive_expect_tx(full, kv ? code_bytes : code_bytes + 2u * (uint32_t)(rows16[0] + rows16[1]) * 4u + q_bytes);
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (rows16[t] == 0) continue;
+                        const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
+                        const uint32_t dst = sl + (kv ? L::kV : L::kK) + t * 16384;
+                        if (rows16[t] == kStTile) {
+                            tc::tma_load_2d(dst, &map_tile, 0, row0, full);
+                        } else {
+                            for (int r = 0; r < rows16[t]; r += kStTailBox)
+                                tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
+                        }
+                        if (kv == 0) {
+                            tc::bulk_load(sl + L::kKs + t * 512, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
+                                          (uint32_t)rows16[t] * 4u, full);
+                            tc::bulk_load(sl + L::kVs + t * 512, p.scales + scale_block_offset(page[t], chead, 1, p.Hkv),
+                                          (uint32_t)rows16[t] * 4u, full);
+                        }
+                    }
+                    if (kv == 0)
+                        tc::bulk_load(sl + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes, full);
+                }
+            }
+        }
+    } else {
+        // =========================================================== consumers: thread = token (tile 0: gtid, tile 1: 128 + gtid)
+        const int g = warp >> 2, gtid = tid & 127, gw = warp & 3;
+        unsigned char *grp = smem + L::kGroup0 + g * L::kGroupBytes;
+        float *red_m = reinterpret_cast<float *>(grp + L::kRed);   // [NH][4]
+        float *red_l = red_m + 4 * NH;                             // [NH][4]
+        float *rowscale = red_l + 4 * NH;                          // [NH]
+        const uint32_t qop_addr = sbase + L::kGroup0 + g * L::kGroupBytes + L::kQop;
+        const uint32_t tm = tmem + (uint32_t)g * 128u;             // this group's columns: S tile 0 | S tile 1 | O
+        const uint32_t lane_base = (uint32_t)(gw * 32) << 16;
+        const int bar_id = 1 + g;
+
+        for (int n = g; n < cnt; n += kStGroups) {
+            const int slot = n % kStSlots;
+            const uint32_t ph = (uint32_t)(n / kStSlots) & 1u;
+            const uint32_t mph = (uint32_t)(n / kStGroups) & 1u;
+            unsigned char *sl = smem + slot * L::kSlotBytes;
+            const uint32_t sl_addr = sbase + slot * L::kSlotBytes;
+            wait(bar_full_k(slot), ph);
+            const int4 meta = *reinterpret_cast<const int4 *>(sl + L::kMeta);
+            const int b = meta.x, head = meta.y, chunk = meta.z, n_tok = meta.w;
+            const int n_tiles = n_tok > kStTile ? 2 : 1;
+            const int h0 = head * p.G;
+
+            // ---- query operand: warp w converts heads w, w+4, ...; a lane owns four consecutive dims
+            for (int h = gw; h < p.G; h += 4) {
+                const uint2 raw = *reinterpret_cast<const uint2 *>(sl + L::kQraw + h * 256 + lane * 8);
+                const float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
+                                    bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
+                const float am = warp_max(fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
+                const float p2 = pow2_floor(am);
+                const float f = pow2_recip(p2) * kStQFix;
+                uint32_t lo_w = 0, hi_w = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // v = round(x * f), |v| < 16384, as the low 16 bits of 1.5 * 2^23 + v (two's complement)
+                    const int v = (int)(int16_t)(__float_as_uint(fmaf(x[i], f, 12582912.f)) & 0xFFFFu);
+                    const int hi = (v + 128) >> 8;            // v = 256 * hi + lo with lo in [-128, 127]
+                    lo_w |= ((uint32_t)v & 0xFFu) << (8 * i);
+                    hi_w |= ((uint32_t)hi & 0xFFu) << (8 * i);
+                }
+                if (lane == 0) rowscale[h] = p2 * p.scale_log2e * (1.f / kStQFix);
+                *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(h, 4 * lane)) = hi_w;
+                *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(NH + h, 4 * lane)) = lo_w;
+            }
+            tc::fence_proxy_async();
+            tc::named_barrier(bar_id, kStGroupThreads);
+
+            // ---- scores on the tensor cores
+            if (gtid == 0) {
+                tc::fence_after_sync();
+                constexpr uint32_t idesc = tc::instr_desc(2, 1, 1, false, false, 128, N);   // s32 <- s8 (K-major) x s8 (K-major)
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t a = tc::smem_desc(sl_addr + L::kK + t * 16384 + j * 32, 16, 1024, tc::kSwizzle128B);
+                            const uint64_t bq = tc::smem_desc(qop_addr + j * 256, 128, 1024, tc::kSwizzleNone);
+                            tc::mma_i8(tm + t * N, a, bq, idesc, j > 0);
+                        }
+                    }
+                }
+                tc::commit(bar_mma_s(g));
+            }
+
+            // this thread's two tokens
+            float sk[2], lsv[2], rsv[2];
+            bool valid[2];
+            {
+                const float *ks_s = reinterpret_cast<const float *>(sl + L::kKs);
+                const float *vs_s = reinterpret_cast<const float *>(sl + L::kVs);
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const int tok = t * kStTile + gtid;
+                    valid[t] = tok < n_tok;
+                    const float sv = valid[t] ? fmaxf(vs_s[tok], kMinScale) : 1.f;
+                    sk[t] = valid[t] ? ks_s[tok] : 0.f;
+                    lsv[t] = __log2f(sv);
+                    rsv[t] = valid[t] ? __frcp_rn(sv) : 0.f;
+                }
+            }
+
+            wait(bar_mma_s(g), mph);
+            __syncwarp();   // reconverge after the wait loop: the tensor-memory loads below are warp-aligned
+            tc::fence_after_sync();
+
+            // ---- S^T from tensor memory: row = token, columns [hi | lo] per head
+            float s[2][NH];
+            float mloc[NH];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) mloc[h] = -INFINITY;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                if (t < n_tiles) {
+                    uint32_t r[N];
+#pragma unroll
+                    for (int c16 = 0; c16 < N / 16; ++c16) {
+                        uint32_t tmp[16];
+                        tc::tmem_ld16(tm + lane_base + t * N + c16 * 16, tmp);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) r[c16 * 16 + i] = tmp[i];
+                    }
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) {
+                        const float x = (float)(((int)r[h] << 8) + (int)r[NH + h]);
+                        s[t][h] = (valid[t] && h < p.G) ? fmaf(x, sk[t] * rowscale[h], lsv[t]) : -INFINITY;
+                        mloc[h] = fmaxf(mloc[h], s[t][h]);
+                    }
+                } else {
+#pragma unroll
+                    for (int h = 0; h < NH; ++h) s[t][h] = -INFINITY;
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (h < p.G) {
+                    const float m = warp_max(mloc[h]);
+                    if (lane == 0) red_m[h * 4 + gw] = m;
+                }
+            }
+            tc::fence_before_sync();
+            tc::named_barrier(bar_id, kStGroupThreads);
+
+            // ---- one softmax over the chunk's scores per head; P^T (bytes [hi | lo]) into K tile 0
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (h < p.G) {
+                    const float4 mw = *reinterpret_cast<const float4 *>(red_m + h * 4);
+                    const float M = fmaxf(fmaxf(mw.x, mw.y), fmaxf(mw.z, mw.w));
+                    float lloc = 0.f;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (t < n_tiles) {
+                            const float e = exp2f(s[t][h] - M);
+                            lloc = fmaf(e, rsv[t], lloc);
+                            const uint32_t bits = __float_as_uint(fmaf(e, kStPFix, 8388608.f));   // 2^23 + round(e * 65535)
+                            unsigned char *pt = sl + L::kK + t * L::kPTileBytes;
+                            pt[st_core_off(h, gtid)] = (unsigned char)((bits >> 8) & 0xFFu);
+                            pt[st_core_off(NH + h, gtid)] = (unsigned char)(bits & 0xFFu);
+                        }
+                    }
+                    const float l = warp_sum(lloc);
+                    if (lane == 0) red_l[h * 4 + gw] = l;
+                }
+            }
+            tc::fence_proxy_async();
+            tc::named_barrier(bar_id, kStGroupThreads);
+
+            // ---- O^T = V^T . P^T on the tensor cores
+            if (gtid == 0) {
+                wait(bar_full_v(slot), ph);
+                tc::fence_after_sync();
+                constexpr uint32_t idesc = tc::instr_desc(2, 1, 0, true, false, 128, N);   // s32 <- s8 (MN-major) x u8 (K-major)
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t a = tc::smem_desc(sl_addr + L::kV + t * 16384 + j * 4096, 1024, 1024, tc::kSwizzle128B);
+                            const uint64_t bp = tc::smem_desc(sl_addr + L::kK + t * L::kPTileBytes + j * 256, 128, 1024, tc::kSwizzleNone);
+                            tc::mma_i8(tm + 2 * N, a, bp, idesc, (t > 0) || (j > 0));
+                        }
+                    }
+                }
+                tc::commit(bar_mma_pv(g));
+            }
+            wait(bar_mma_pv(g), mph);
+            __syncwarp();
+            tc::fence_after_sync();
+            // the tensor cores have read the slot for the last time; every generic read of it happened before the barriers above
+            if (gtid == 0) tc::mbar_arrive(bar_empty(slot));
+
+            // ---- O^T from tensor memory: row = head dim, columns [hi | lo] per head; one partial per head
+            {
+                uint32_t r[N];
+#pragma unroll
+                for (int c16 = 0; c16 < N / 16; ++c16) {
+                    uint32_t tmp[16];
+                    tc::tmem_ld16(tm + lane_base + 2 * N + c16 * 16, tmp);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[c16 * 16 + i] = tmp[i];
+                }
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int h = 0; h < NH; ++h) {
+                    if (h < p.G) {
+                        const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_chunks + chunk;
+                        p.part_o[ps * kHeadDim + gtid] = (float)(((int)r[h] << 8) + (int)r[NH + h]) * (1.f / kStPFix);
+                    }
+                }
+            }
+            if (gtid < p.G) {
+                const size_t ps = ((size_t)b * p.Hq + h0 + gtid) * p.n_chunks + chunk;
+                const float4 mw = *reinterpret_cast<const float4 *>(red_m + gtid * 4);
+                const float4 lw = *reinterpret_cast<const float4 *>(red_l + gtid * 4);
+                p.part_ml[ps * 2] = fmaxf(fmaxf(mw.x, mw.y), fmaxf(mw.z, mw.w));
+                p.part_ml[ps * 2 + 1] = (lw.x + lw.y) + (lw.z + lw.w);
+            }
+            // the next chunk's MMAs overwrite this group's tensor-memory columns: the loads above have retired
+            tc::fence_before_sync();
+        }
+    }
+
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 8) {
+        if (lane == 0 && *fail != 0) {
+            // a wait ran out somewhere: give the copies still in flight a bounded chance to land before the block exits
+            for (int n = max(0, cnt - kStSlots); n < cnt; ++n) {
+                const int slot = n % kStSlots;
+                const uint32_t ph = (uint32_t)(n / kStSlots) & 1u;
+                tc::mbar_wait(bar_full_k(slot), ph, 1u << 14);
+                tc::mbar_wait(bar_full_v(slot), ph, 1u << 14);
+            }
+            if (p.status != nullptr) atomicExch(p.status, SLIM_ERR_TIMEOUT);
+        }
+        __syncwarp();
+        tc::fence_after_sync();
+        tc::tmem_dealloc(tmem, kStTmemCols);
+    }
+}
+
+int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int B, cudaStream_t stream)
+{
+    CUtensorMap map_tile, map_tail;
+    int rc = codes_tensor_map(c, kStTile, &map_tile);
+    if (rc != SLIM_OK) return rc;
+    rc = codes_tensor_map(c, kStTailBox, &map_tail);
+    if (rc != SLIM_OK) return rc;
+    int sms = 0;
+    rc = sm_count(&sms);
+    if (rc != SLIM_OK) return rc;
+    const long long max_items = (long long)p.n_chunks * p.Hkv * B;
+    const unsigned grid = (unsigned)(max_items < sms ? max_items : sms);
+    if (p.G <= 8) {
+        constexpr int bytes = (int)StSmem<8>::kBytes;
+        SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        slim_decode_stream_kernel<8><<<grid, kStThreads, bytes, stream>>>(map_tile, map_tail, p, B);
+    } else {
+        constexpr int bytes = (int)StSmem<16>::kBytes;
+        SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        slim_decode_stream_kernel<16><<<grid, kStThreads, bytes, stream>>>(map_tile, map_tail, p, B);
+    }
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}
+
+}  // namespace slim
