@@ -7,9 +7,12 @@
 //  * One thread block per SM.  The work - every 256-token chunk of every (sequence, kv head) - is cut
 //    into one contiguous range per block.  A chunk is the unit of a partial result (m, l, O[128]).
 //  * Warp 8 is the producer: one thread walks the block's chunks and asks the TMA engine for each
-//    chunk's INT8 K tiles, V tiles, scales and query rows into a ring of three shared-memory slots
-//    (128-byte swizzled tiles, completion counted on mbarriers).  A ragged last tile is fetched in
-//    16-row boxes so that no byte beyond the chunk's tokens (rounded up to 16) is read.
+//    chunk's INT8 K tiles and V tiles into a ring of 16 KB tile stages (128-byte swizzled, completion
+//    counted on mbarriers) and for its scales and query rows into a small ring of chunk records.  A
+//    stage goes back to the producer the moment the tensor cores have read it (the MMA completion
+//    itself arrives on the stage's mbarrier), so K tiles are held only until the scores are out and
+//    most of the ring is in flight at any time.  A ragged last tile is fetched in 16-row boxes so
+//    that no byte beyond the chunk's tokens (rounded up to 16) is read.
 //  * Warps 0-3 and 4-7 are two consumer groups that take chunks alternately.  For its chunk a group
 //      - builds the query operand: a 14-bit fixed-point copy of the G = Hq/Hkv query rows of the kv
 //        head, two signed bytes per value (columns [high bytes | low bytes]);
@@ -37,10 +40,11 @@ namespace slim {
 constexpr int kStGroups = 2;
 constexpr int kStGroupThreads = 128;
 constexpr int kStThreads = kStGroups * kStGroupThreads + 32;   // two consumer groups + the producer warp
-constexpr int kStSlots = 3;
+constexpr int kStInfoSlots = 4;                                 // chunk records in flight
 constexpr int kStTile = 128;                                    // tokens per MMA tile (= one page)
 constexpr int kStChunk = 2 * kStTile;                           // tokens per chunk / partial
 constexpr int kStTailBox = 16;                                  // rows per TMA box of a ragged tile
+constexpr uint32_t kStTileBytes = kStTile * kHeadDim;           // 16 KB
 constexpr float kStQFix = 8192.f;      // |q / pow2| < 2  ->  |v| < 16384, high byte in [-64, 64]
 constexpr float kStPFix = 65535.f;
 constexpr uint32_t kStTmemCols = 256;  // 128 per group: S of two tiles + O
@@ -50,27 +54,29 @@ static_assert(kStChunk == 256, "partials are indexed by 256-token chunks (decode
 template <int NH>
 struct StSmem {
     static constexpr int N = 2 * NH;                        // MMA columns: [hi bytes of NH heads | lo bytes]
-    // one ring slot = one chunk
-    static constexpr uint32_t kK = 0;                       // two K tiles, 16 KB each
-    static constexpr uint32_t kV = 32768;                   // two V tiles
-    static constexpr uint32_t kKs = 65536;                  // 256 K scales
-    static constexpr uint32_t kVs = kKs + 1024;             // 256 V scales
-    static constexpr uint32_t kQraw = kVs + 1024;           // the kv head's query rows, bf16 [G][128]
-    static constexpr uint32_t kMeta = kQraw + NH * 256;     // int4: sequence, kv head, chunk, valid tokens
-    static constexpr uint32_t kSlotBytes = (kMeta + 16 + 1023) / 1024 * 1024;
-    static constexpr uint32_t kPTileBytes = N * 128;        // a P^T tile (aliases K tile 0 once the scores are out)
+    static constexpr int kStages = (NH <= 8) ? 12 : 11;     // tile stages of the ring
+    // chunk record: both scale vectors, the kv head's query rows, the chunk's coordinates
+    static constexpr uint32_t kKs = 0;                      // 256 K scales
+    static constexpr uint32_t kVs = 1024;                   // 256 V scales
+    static constexpr uint32_t kQraw = 2048;                 // bf16 [G][128]
+    static constexpr uint32_t kMeta = kQraw + NH * 256;     // int[5]: sequence, kv head, chunk, valid tokens, first tile index
+    static constexpr uint32_t kInfoBytes = (kMeta + 32 + 127) / 128 * 128;
+    static constexpr uint32_t kInfo0 = kStages * kStTileBytes;
     // per consumer group
-    static constexpr uint32_t kGroup0 = kStSlots * kSlotBytes;
-    static constexpr uint32_t kQop = 0;                     // query operand: N rows x 128 bytes, core-matrix layout
-    static constexpr uint32_t kRed = N * 128;               // floats: [NH][4] warp maxima, [NH][4] warp sums, [NH] row scales
+    static constexpr uint32_t kGroup0 = kInfo0 + kStInfoSlots * kInfoBytes;
+    static constexpr uint32_t kPTileBytes = N * 128;        // a P^T tile, core-matrix layout
+    static constexpr uint32_t kP = 0;                       // two P^T tiles
+    static constexpr uint32_t kQop = 2 * kPTileBytes;       // query operand: N rows x 128 bytes, core-matrix layout
+    static constexpr uint32_t kRed = kQop + N * 128;        // floats: [NH][4] warp maxima, [NH][4] warp sums, [NH] row scales
     static constexpr uint32_t kGroupBytes = (kRed + 9 * NH * 4 + 127) / 128 * 128;
-    // block-wide
-    static constexpr uint32_t kBar = kGroup0 + kStGroups * kGroupBytes;   // 13 mbarriers
-    static constexpr uint32_t kTmemSlot = kBar + 13 * 8;
-    static constexpr uint32_t kRange = kTmemSlot + 8;       // int[4]: chunks of this block, first sequence / head / chunk
+    // block-wide: mbarriers full[kStages], empty[kStages], info full[4], info empty[4], S done[2], PV done[2]
+    static constexpr uint32_t kBar = kGroup0 + kStGroups * kGroupBytes;
+    static constexpr int kNumBars = 2 * kStages + 2 * kStInfoSlots + 2 * kStGroups;
+    static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
+    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[4]: chunks of this block, first sequence / head / chunk
     static constexpr uint32_t kFail = kRange + 16;
     static constexpr uint32_t kBytes = kFail + 8;
-    static_assert(2 * kPTileBytes <= 16384, "both P^T tiles live in K tile 0");
+    static_assert(kRange % 16 == 0, "range record is read as int4-aligned ints");
     static_assert(kBytes <= 232448, "shared memory budget of one block");
 };
 
@@ -95,21 +101,23 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 {
     using L = StSmem<NH>;
     constexpr int N = L::N;
+    constexpr int S = L::kStages;
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + L::kBar;
-    auto bar_full_k = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-    auto bar_full_v = [&](int s) { return bar0 + 8u * (uint32_t)(3 + s); };
-    auto bar_empty = [&](int s) { return bar0 + 8u * (uint32_t)(6 + s); };
-    auto bar_mma_s = [&](int g) { return bar0 + 8u * (uint32_t)(9 + g); };
-    auto bar_mma_pv = [&](int g) { return bar0 + 8u * (uint32_t)(11 + g); };
+    auto bar_full = [&](int st) { return bar0 + 8u * (uint32_t)st; };
+    auto bar_empty = [&](int st) { return bar0 + 8u * (uint32_t)(S + st); };
+    auto bar_info_full = [&](int i) { return bar0 + 8u * (uint32_t)(2 * S + i); };
+    auto bar_info_empty = [&](int i) { return bar0 + 8u * (uint32_t)(2 * S + kStInfoSlots + i); };
+    auto bar_mma_s = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + g); };
+    auto bar_mma_pv = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + kStGroups + g); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kTmemSlot);
     int *range = reinterpret_cast<int *>(smem + L::kRange);
     volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
 
     if (tid == 0) {
-        for (int i = 0; i < 13; ++i) tc::mbar_init(bar0 + 8u * i, 1);
+        for (int i = 0; i < L::kNumBars; ++i) tc::mbar_init(bar0 + 8u * i, 1);
         tc::mbar_init_fence();
         *fail = 0;
     }
@@ -175,6 +183,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             *fail = 1;
         }
     };
+    int tiles_issued = 0;   // producer thread: tile stages armed so far (ring position)
 
     if (warp == 8) {
         // =========================================================== producer (one thread)
@@ -190,9 +199,11 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 return r;
             };
             int2 pg = page_ids(b, chunk);
+            int stage = 0;
+            uint32_t stage_ph = 0;   // parity of the stage's current use
             for (int n = 0; n < cnt; ++n) {
-                const int slot = n % kStSlots;
-                const uint32_t ph = (uint32_t)(n / kStSlots) & 1u;
+                const int islot = n % kStInfoSlots;
+                const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
                 const int cb = b, chead = head, cchunk = chunk;
                 const int n_tok = min(kStChunk, len - chunk * kStChunk);
                 const int2 cpg = pg;
@@ -211,9 +222,6 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     }
                     pg = page_ids(min(b, B - 1), chunk);
                 }
-                wait(bar_empty(slot), ph ^ 1u);
-                const uint32_t sl = sbase + slot * L::kSlotBytes;
-                *reinterpret_cast<int4 *>(smem + slot * L::kSlotBytes + L::kMeta) = make_int4(cb, chead, cchunk, n_tok);
                 int page[2] = {cpg.x, cpg.y};
                 int rows16[2];
 #pragma unroll
@@ -222,33 +230,47 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const int rows = max(0, min(kStTile, n_tok - t * kStTile));
                     rows16[t] = (rows + kStTailBox - 1) / kStTailBox * kStTailBox;
                 }
-                const uint32_t code_bytes = (uint32_t)(rows16[0] + rows16[1]) * kHeadDim;
+                // ---- the chunk record: coordinates, both scale vectors, the query rows
+                wait(bar_info_empty(islot), iph ^ 1u);
+                unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
+                const uint32_t info_addr = sbase + L::kInfo0 + islot * L::kInfoBytes;
+                int *meta = reinterpret_cast<int *>(info + L::kMeta);
+                meta[0] = cb, meta[1] = chead, meta[2] = cchunk, meta[3] = n_tok, meta[4] = tiles_issued;
                 const uint32_t q_bytes = (uint32_t)p.G * kHeadDim * 2u;
+                tc::mbar_arrive_expect_tx(bar_info_full(islot), 2u * (uint32_t)(rows16[0] + rows16[1]) * 4u + q_bytes);
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (rows16[t] == 0) continue;
+                    tc::bulk_load(info_addr + L::kKs + t * 512, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
+                                  (uint32_t)rows16[t] * 4u, bar_info_full(islot));
+                    tc::bulk_load(info_addr + L::kVs + t * 512, p.scales + scale_block_offset(page[t], chead, 1, p.Hkv),
+                                  (uint32_t)rows16[t] * 4u, bar_info_full(islot));
+                }
+                tc::bulk_load(info_addr + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes,
+                              bar_info_full(islot));
+                // ---- the chunk's tiles, in the order the consumers need them: K tiles, then V tiles
 #pragma unroll
                 for (int kv = 0; kv < 2; ++kv) {
-                    const uint32_t full = kv ? bar_full_v(slot) : bar_full_k(slot);
-                    // K barrier: K tiles + both scale vectors + the query rows; V barrier: V tiles
-                    tc::mbar_arrive_expect_tx(full, kv ? code_bytes : code_bytes + 2u * (uint32_t)(rows16[0] + rows16[1]) * 4u + q_bytes);
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         if (rows16[t] == 0) continue;
+                        wait(bar_empty(stage), stage_ph ^ 1u);
+                        const uint32_t full = bar_full(stage);
+                        tc::mbar_arrive_expect_tx(full, (uint32_t)rows16[t] * kHeadDim);
                         const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
-                        const uint32_t dst = sl + (kv ? L::kV : L::kK) + t * 16384;
+                        const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
                         if (rows16[t] == kStTile) {
                             tc::tma_load_2d(dst, &map_tile, 0, row0, full);
                         } else {
                             for (int r = 0; r < rows16[t]; r += kStTailBox)
                                 tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
                         }
-                        if (kv == 0) {
-                            tc::bulk_load(sl + L::kKs + t * 512, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
-                                          (uint32_t)rows16[t] * 4u, full);
-                            tc::bulk_load(sl + L::kVs + t * 512, p.scales + scale_block_offset(page[t], chead, 1, p.Hkv),
-                                          (uint32_t)rows16[t] * 4u, full);
+                        ++tiles_issued;
+                        if (++stage == S) {
+                            stage = 0;
+                            stage_ph ^= 1u;
                         }
                     }
-                    if (kv == 0)
-                        tc::bulk_load(sl + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes, full);
                 }
             }
         }
@@ -259,26 +281,25 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         float *red_m = reinterpret_cast<float *>(grp + L::kRed);   // [NH][4]
         float *red_l = red_m + 4 * NH;                             // [NH][4]
         float *rowscale = red_l + 4 * NH;                          // [NH]
-        const uint32_t qop_addr = sbase + L::kGroup0 + g * L::kGroupBytes + L::kQop;
+        const uint32_t grp_addr = sbase + L::kGroup0 + g * L::kGroupBytes;
         const uint32_t tm = tmem + (uint32_t)g * 128u;             // this group's columns: S tile 0 | S tile 1 | O
         const uint32_t lane_base = (uint32_t)(gw * 32) << 16;
         const int bar_id = 1 + g;
 
         for (int n = g; n < cnt; n += kStGroups) {
-            const int slot = n % kStSlots;
-            const uint32_t ph = (uint32_t)(n / kStSlots) & 1u;
+            const int islot = n % kStInfoSlots;
+            const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
             const uint32_t mph = (uint32_t)(n / kStGroups) & 1u;
-            unsigned char *sl = smem + slot * L::kSlotBytes;
-            const uint32_t sl_addr = sbase + slot * L::kSlotBytes;
-            wait(bar_full_k(slot), ph);
-            const int4 meta = *reinterpret_cast<const int4 *>(sl + L::kMeta);
-            const int b = meta.x, head = meta.y, chunk = meta.z, n_tok = meta.w;
+            const unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
+            wait(bar_info_full(islot), iph);
+            const int *meta = reinterpret_cast<const int *>(info + L::kMeta);
+            const int b = meta[0], head = meta[1], chunk = meta[2], n_tok = meta[3], tile0 = meta[4];
             const int n_tiles = n_tok > kStTile ? 2 : 1;
             const int h0 = head * p.G;
 
             // ---- query operand: warp w converts heads w, w+4, ...; a lane owns four consecutive dims
             for (int h = gw; h < p.G; h += 4) {
-                const uint2 raw = *reinterpret_cast<const uint2 *>(sl + L::kQraw + h * 256 + lane * 8);
+                const uint2 raw = *reinterpret_cast<const uint2 *>(info + L::kQraw + h * 256 + lane * 8);
                 const float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
                                     bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
                 const float am = warp_max(fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
@@ -297,33 +318,12 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(h, 4 * lane)) = hi_w;
                 *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(NH + h, 4 * lane)) = lo_w;
             }
-            tc::fence_proxy_async();
-            tc::named_barrier(bar_id, kStGroupThreads);
-
-            // ---- scores on the tensor cores
-            if (gtid == 0) {
-                tc::fence_after_sync();
-                constexpr uint32_t idesc = tc::instr_desc(2, 1, 1, false, false, 128, N);   // s32 <- s8 (K-major) x s8 (K-major)
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t < n_tiles) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t a = tc::smem_desc(sl_addr + L::kK + t * 16384 + j * 32, 16, 1024, tc::kSwizzle128B);
-                            const uint64_t bq = tc::smem_desc(qop_addr + j * 256, 128, 1024, tc::kSwizzleNone);
-                            tc::mma_i8(tm + t * N, a, bq, idesc, j > 0);
-                        }
-                    }
-                }
-                tc::commit(bar_mma_s(g));
-            }
-
             // this thread's two tokens
             float sk[2], lsv[2], rsv[2];
             bool valid[2];
             {
-                const float *ks_s = reinterpret_cast<const float *>(sl + L::kKs);
-                const float *vs_s = reinterpret_cast<const float *>(sl + L::kVs);
+                const float *ks_s = reinterpret_cast<const float *>(info + L::kKs);
+                const float *vs_s = reinterpret_cast<const float *>(info + L::kVs);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     const int tok = t * kStTile + gtid;
@@ -333,6 +333,41 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     lsv[t] = __log2f(sv);
                     rsv[t] = valid[t] ? __frcp_rn(sv) : 0.f;
                 }
+            }
+            tc::fence_proxy_async();
+            tc::named_barrier(bar_id, kStGroupThreads);
+
+            // ---- scores on the tensor cores; each K stage goes back to the producer when the MMAs have read it
+            if (gtid == 0) {
+                // every thread of the group has read the chunk record (scales, query rows, coordinates)
+                tc::mbar_arrive(bar_info_empty(islot));
+                constexpr uint32_t idesc = tc::instr_desc(2, 1, 1, false, false, 128, N);   // s32 <- s8 (K-major) x s8 (K-major)
+                int kst[2];
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+                        const int gi = tile0 + t;
+                        kst[t] = gi % S;
+                        wait(bar_full(kst[t]), (uint32_t)(gi / S) & 1u);
+                    }
+                }
+                tc::fence_after_sync();
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+                        const uint32_t k_addr = sbase + (uint32_t)kst[t] * kStTileBytes;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t a = tc::smem_desc(k_addr + j * 32, 16, 1024, tc::kSwizzle128B);
+                            const uint64_t bq = tc::smem_desc(grp_addr + L::kQop + j * 256, 128, 1024, tc::kSwizzleNone);
+                            tc::mma_i8(tm + t * N, a, bq, idesc, j > 0);
+                        }
+                    }
+                }
+                tc::commit(bar_mma_s(g));
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles) tc::commit(bar_empty(kst[t]));
             }
 
             wait(bar_mma_s(g), mph);
@@ -377,7 +412,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             tc::fence_before_sync();
             tc::named_barrier(bar_id, kStGroupThreads);
 
-            // ---- one softmax over the chunk's scores per head; P^T (bytes [hi | lo]) into K tile 0
+            // ---- one softmax over the chunk's scores per head; P^T as bytes [hi | lo]
 #pragma unroll
             for (int h = 0; h < NH; ++h) {
                 if (h < p.G) {
@@ -390,7 +425,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                             const float e = exp2f(s[t][h] - M);
                             lloc = fmaf(e, rsv[t], lloc);
                             const uint32_t bits = __float_as_uint(fmaf(e, kStPFix, 8388608.f));   // 2^23 + round(e * 65535)
-                            unsigned char *pt = sl + L::kK + t * L::kPTileBytes;
+                            unsigned char *pt = grp + L::kP + t * L::kPTileBytes;
                             pt[st_core_off(h, gtid)] = (unsigned char)((bits >> 8) & 0xFFu);
                             pt[st_core_off(NH + h, gtid)] = (unsigned char)(bits & 0xFFu);
                         }
@@ -402,29 +437,39 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             tc::fence_proxy_async();
             tc::named_barrier(bar_id, kStGroupThreads);
 
-            // ---- O^T = V^T . P^T on the tensor cores
+            // ---- O^T = V^T . P^T on the tensor cores; the V stages go back when the MMAs have read them
             if (gtid == 0) {
-                wait(bar_full_v(slot), ph);
-                tc::fence_after_sync();
                 constexpr uint32_t idesc = tc::instr_desc(2, 1, 0, true, false, 128, N);   // s32 <- s8 (MN-major) x u8 (K-major)
+                int vst[2];
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (t < n_tiles) {
+                        const int gi = tile0 + n_tiles + t;
+                        vst[t] = gi % S;
+                        wait(bar_full(vst[t]), (uint32_t)(gi / S) & 1u);
+                    }
+                }
+                tc::fence_after_sync();
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+                        const uint32_t v_addr = sbase + (uint32_t)vst[t] * kStTileBytes;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const uint64_t a = tc::smem_desc(sl_addr + L::kV + t * 16384 + j * 4096, 1024, 1024, tc::kSwizzle128B);
-                            const uint64_t bp = tc::smem_desc(sl_addr + L::kK + t * L::kPTileBytes + j * 256, 128, 1024, tc::kSwizzleNone);
+                            const uint64_t a = tc::smem_desc(v_addr + j * 4096, 1024, 1024, tc::kSwizzle128B);
+                            const uint64_t bp = tc::smem_desc(grp_addr + L::kP + t * L::kPTileBytes + j * 256, 128, 1024, tc::kSwizzleNone);
                             tc::mma_i8(tm + 2 * N, a, bp, idesc, (t > 0) || (j > 0));
                         }
                     }
                 }
                 tc::commit(bar_mma_pv(g));
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles) tc::commit(bar_empty(vst[t]));
             }
             wait(bar_mma_pv(g), mph);
             __syncwarp();
             tc::fence_after_sync();
-            // the tensor cores have read the slot for the last time; every generic read of it happened before the barriers above
-            if (gtid == 0) tc::mbar_arrive(bar_empty(slot));
 
             // ---- O^T from tensor memory: row = head dim, columns [hi | lo] per head; one partial per head
             {
@@ -462,12 +507,10 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     if (warp == 8) {
         if (lane == 0 && *fail != 0) {
             // a wait ran out somewhere: give the copies still in flight a bounded chance to land before the block exits
-            for (int n = max(0, cnt - kStSlots); n < cnt; ++n) {
-                const int slot = n % kStSlots;
-                const uint32_t ph = (uint32_t)(n / kStSlots) & 1u;
-                tc::mbar_wait(bar_full_k(slot), ph, 1u << 14);
-                tc::mbar_wait(bar_full_v(slot), ph, 1u << 14);
-            }
+            for (int gi = max(0, tiles_issued - S); gi < tiles_issued; ++gi)
+                tc::mbar_wait(bar_full(gi % S), (uint32_t)(gi / S) & 1u, 1u << 14);
+            for (int n = max(0, cnt - kStInfoSlots); n < cnt; ++n)
+                tc::mbar_wait(bar_info_full(n % kStInfoSlots), (uint32_t)(n / kStInfoSlots) & 1u, 1u << 14);
             if (p.status != nullptr) atomicExch(p.status, SLIM_ERR_TIMEOUT);
         }
         __syncwarp();
