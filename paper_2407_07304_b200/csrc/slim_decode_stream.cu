@@ -13,6 +13,9 @@
 //    itself arrives on the stage's mbarrier), so K tiles are held only until the scores are out and
 //    most of the ring is in flight at any time.  A ragged last tile is fetched in 16-row boxes so
 //    that no byte beyond the chunk's tokens (rounded up to 16) is read.
+//  * Warps 9 and 10 each hold one MMA-issuing thread, one per consumer group: it waits for the chunk's
+//    tiles and for the group's operands, issues the tcgen05.mma instructions and commits their
+//    completion to the group's mbarrier and to the stages' "empty" mbarriers.
 //  * Warps 0-3 and 4-7 are two consumer groups that take chunks alternately.  For its chunk a group
 //      - builds the query operand: a 14-bit fixed-point copy of the G = Hq/Hkv query rows of the kv
 //        head, two signed bytes per value (columns [high bytes | low bytes]);
@@ -39,7 +42,7 @@ namespace slim {
 
 constexpr int kStGroups = 2;
 constexpr int kStGroupThreads = 128;
-constexpr int kStThreads = kStGroups * kStGroupThreads + 32;   // two consumer groups + the producer warp
+constexpr int kStThreads = kStGroups * kStGroupThreads + 32 + kStGroups * 32;   // consumer groups + producer warp + one MMA-issue warp per group
 constexpr int kStInfoSlots = 4;                                 // chunk records in flight
 constexpr int kStTile = 128;                                    // tokens per MMA tile (= one page)
 constexpr int kStChunk = 2 * kStTile;                           // tokens per chunk / partial
@@ -54,7 +57,7 @@ static_assert(kStChunk == 256, "partials are indexed by 256-token chunks (decode
 template <int NH>
 struct StSmem {
     static constexpr int N = 2 * NH;                        // MMA columns: [hi bytes of NH heads | lo bytes]
-    static constexpr int kStages = (NH <= 8) ? 12 : 11;     // tile stages of the ring
+    static constexpr int kStages = (NH <= 8) ? 11 : 10;     // tile stages of the ring
     // chunk record: both scale vectors, the kv head's query rows, the chunk's coordinates
     static constexpr uint32_t kKs = 0;                      // 256 K scales
     static constexpr uint32_t kVs = 1024;                   // 256 V scales
@@ -67,11 +70,13 @@ struct StSmem {
     static constexpr uint32_t kPTileBytes = N * 128;        // a P^T tile, core-matrix layout
     static constexpr uint32_t kP = 0;                       // two P^T tiles
     static constexpr uint32_t kQop = 2 * kPTileBytes;       // query operand: N rows x 128 bytes, core-matrix layout
-    static constexpr uint32_t kRed = kQop + N * 128;        // floats: [NH][4] warp maxima, [NH][4] warp sums, [NH] row scales
-    static constexpr uint32_t kGroupBytes = (kRed + 9 * NH * 4 + 127) / 128 * 128;
-    // block-wide: mbarriers full[kStages], empty[kStages], info full[4], info empty[4], S done[2], PV done[2]
+    static constexpr uint32_t kLsum = kQop + N * 128;       // floats [NH][128]: every token thread's share of the softmax denominators
+    static constexpr uint32_t kRed = kLsum + NH * 512;      // floats: [NH][4] warp maxima, [NH] row scales
+    static constexpr uint32_t kGroupBytes = (kRed + 5 * NH * 4 + 127) / 128 * 128;
+    // block-wide: mbarriers full[kStages], empty[kStages], info full[4], info empty[4],
+    //             operands ready for S[2], for PV[2], S done[2], PV done[2]
     static constexpr uint32_t kBar = kGroup0 + kStGroups * kGroupBytes;
-    static constexpr int kNumBars = 2 * kStages + 2 * kStInfoSlots + 2 * kStGroups;
+    static constexpr int kNumBars = 2 * kStages + 2 * kStInfoSlots + 4 * kStGroups;
     static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
     static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[4]: chunks of this block, first sequence / head / chunk
     static constexpr uint32_t kFail = kRange + 16;
@@ -85,6 +90,30 @@ struct StSmem {
 __device__ __forceinline__ uint32_t st_core_off(int n, int kb)
 {
     return (uint32_t)((n >> 3) * 1024 + (kb >> 4) * 128 + (n & 7) * 16 + (kb & 15));
+}
+
+__device__ __forceinline__ float st_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float st_rcp(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+// Order-preserving map between floats and signed integers (its own inverse), so that an integer
+// warp reduction finds a floating-point maximum.
+__device__ __forceinline__ int st_ordered_int(float x)
+{
+    const int i = __float_as_int(x);
+    return i ^ ((i >> 31) & 0x7FFFFFFF);
+}
+__device__ __forceinline__ float st_ordered_float(int i)
+{
+    return __int_as_float(i ^ ((i >> 31) & 0x7FFFFFFF));
 }
 
 // A sequence's cached tokens, never beyond the page table or the launch's max_kv.
@@ -110,14 +139,30 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     auto bar_empty = [&](int st) { return bar0 + 8u * (uint32_t)(S + st); };
     auto bar_info_full = [&](int i) { return bar0 + 8u * (uint32_t)(2 * S + i); };
     auto bar_info_empty = [&](int i) { return bar0 + 8u * (uint32_t)(2 * S + kStInfoSlots + i); };
-    auto bar_mma_s = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + g); };
-    auto bar_mma_pv = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + kStGroups + g); };
+    auto bar_ready_s = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + g); };
+    auto bar_ready_pv = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + kStGroups + g); };
+    auto bar_mma_s = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + 2 * kStGroups + g); };
+    auto bar_mma_pv = [&](int g) { return bar0 + 8u * (uint32_t)(2 * S + 2 * kStInfoSlots + 3 * kStGroups + g); };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kTmemSlot);
     int *range = reinterpret_cast<int *>(smem + L::kRange);
     volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
 
     if (tid == 0) {
-        for (int i = 0; i < L::kNumBars; ++i) tc::mbar_init(bar0 + 8u * i, 1);
+        for (int i = 0; i < S; ++i) {
+            tc::mbar_init(bar_full(i), 1);
+            tc::mbar_init(bar_empty(i), 1);
+        }
+        for (int i = 0; i < kStInfoSlots; ++i) {
+            tc::mbar_init(bar_info_full(i), 1);
+            // a chunk record is released by the 128 threads of its group and that group's MMA thread
+            tc::mbar_init(bar_info_empty(i), kStGroupThreads + 1);
+        }
+        for (int g = 0; g < kStGroups; ++g) {
+            tc::mbar_init(bar_ready_s(g), kStGroupThreads);
+            tc::mbar_init(bar_ready_pv(g), kStGroupThreads);
+            tc::mbar_init(bar_mma_s(g), 1);
+            tc::mbar_init(bar_mma_pv(g), 1);
+        }
         tc::mbar_init_fence();
         *fail = 0;
     }
@@ -164,7 +209,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             range[2] = head0;
             range[3] = chunk0;
         }
-    } else {
+    } else if (warp < 8) {
         // rows of the query operand that belong to no head stay zero for the whole launch
         const int g = warp >> 2, gtid = tid & 127;
         unsigned char *qop = smem + L::kGroup0 + g * L::kGroupBytes + L::kQop;
@@ -274,17 +319,88 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 }
             }
         }
+    } else if (warp >= 9) {
+        // =========================================================== MMA issue for group g (one thread)
+        const int g = warp - 9;
+        if (lane == 0) {
+            const uint32_t grp_addr = sbase + L::kGroup0 + g * L::kGroupBytes;
+            const uint32_t tm = tmem + (uint32_t)g * 128u;
+            constexpr uint32_t idesc_s = tc::instr_desc(2, 1, 1, false, false, 128, N);    // s32 <- s8 (K-major) x s8 (K-major)
+            constexpr uint32_t idesc_pv = tc::instr_desc(2, 1, 0, true, false, 128, N);    // s32 <- s8 (MN-major) x u8 (K-major)
+            for (int n = g; n < cnt; n += kStGroups) {
+                const int islot = n % kStInfoSlots;
+                const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
+                const uint32_t mph = (uint32_t)(n / kStGroups) & 1u;
+                wait(bar_info_full(islot), iph);
+                const int *meta = reinterpret_cast<const int *>(smem + L::kInfo0 + islot * L::kInfoBytes + L::kMeta);
+                const int n_tok = meta[3], tile0 = meta[4];
+                tc::mbar_arrive(bar_info_empty(islot));
+                const int n_tiles = n_tok > kStTile ? 2 : 1;
+                int st[4];       // stages of K tile 0, K tile 1, V tile 0, V tile 1 (the chunk's tiles in ring order)
+                uint32_t ph[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int gi = tile0 + i;
+                    st[i] = gi % S;
+                    ph[i] = (uint32_t)(gi / S) & 1u;
+                }
+                // ---- scores: S^T[token][head] = K_codes . Q^T; each K stage goes back to the producer when read
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles) wait(bar_full(st[t]), ph[t]);
+                wait(bar_ready_s(g), mph);
+                tc::fence_after_sync();
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+                        const uint32_t k_addr = sbase + (uint32_t)st[t] * kStTileBytes;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t a = tc::smem_desc(k_addr + j * 32, 16, 1024, tc::kSwizzle128B);
+                            const uint64_t bq = tc::smem_desc(grp_addr + L::kQop + j * 256, 128, 1024, tc::kSwizzleNone);
+                            tc::mma_i8(tm + t * N, a, bq, idesc_s, j > 0);
+                        }
+                    }
+                }
+                tc::commit(bar_mma_s(g));
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles) tc::commit(bar_empty(st[t]));
+                // ---- output: O^T[dim][head] = V_codes^T . P^T
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles) wait(bar_full(st[n_tiles + t]), ph[n_tiles + t]);
+                wait(bar_ready_pv(g), mph);
+                tc::fence_after_sync();
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t < n_tiles) {
+                        const uint32_t v_addr = sbase + (uint32_t)st[n_tiles + t] * kStTileBytes;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t a = tc::smem_desc(v_addr + j * 4096, 1024, 1024, tc::kSwizzle128B);
+                            const uint64_t bp = tc::smem_desc(grp_addr + L::kP + t * L::kPTileBytes + j * 256, 128, 1024, tc::kSwizzleNone);
+                            tc::mma_i8(tm + 2 * N, a, bp, idesc_pv, (t > 0) || (j > 0));
+                        }
+                    }
+                }
+                tc::commit(bar_mma_pv(g));
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles) tc::commit(bar_empty(st[n_tiles + t]));
+            }
+        }
     } else {
         // =========================================================== consumers: thread = token (tile 0: gtid, tile 1: 128 + gtid)
         const int g = warp >> 2, gtid = tid & 127, gw = warp & 3;
         unsigned char *grp = smem + L::kGroup0 + g * L::kGroupBytes;
+        float *lsum = reinterpret_cast<float *>(grp + L::kLsum);   // [NH][128]
         float *red_m = reinterpret_cast<float *>(grp + L::kRed);   // [NH][4]
-        float *red_l = red_m + 4 * NH;                             // [NH][4]
-        float *rowscale = red_l + 4 * NH;                          // [NH]
-        const uint32_t grp_addr = sbase + L::kGroup0 + g * L::kGroupBytes;
+        float *rowscale = red_m + 4 * NH;                          // [NH]
         const uint32_t tm = tmem + (uint32_t)g * 128u;             // this group's columns: S tile 0 | S tile 1 | O
         const uint32_t lane_base = (uint32_t)(gw * 32) << 16;
         const int bar_id = 1 + g;
+        int q_b = -1, q_head = -1;                                 // whose query rows the operand buffer holds
 
         for (int n = g; n < cnt; n += kStGroups) {
             const int islot = n % kStInfoSlots;
@@ -293,30 +409,35 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             const unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
             wait(bar_info_full(islot), iph);
             const int *meta = reinterpret_cast<const int *>(info + L::kMeta);
-            const int b = meta[0], head = meta[1], chunk = meta[2], n_tok = meta[3], tile0 = meta[4];
+            const int b = meta[0], head = meta[1], chunk = meta[2], n_tok = meta[3];
             const int n_tiles = n_tok > kStTile ? 2 : 1;
             const int h0 = head * p.G;
 
-            // ---- query operand: warp w converts heads w, w+4, ...; a lane owns four consecutive dims
-            for (int h = gw; h < p.G; h += 4) {
-                const uint2 raw = *reinterpret_cast<const uint2 *>(info + L::kQraw + h * 256 + lane * 8);
-                const float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
-                                    bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
-                const float am = warp_max(fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
-                const float p2 = pow2_floor(am);
-                const float f = pow2_recip(p2) * kStQFix;
-                uint32_t lo_w = 0, hi_w = 0;
+            // ---- query operand (only when the chunk belongs to another (sequence, kv head) than the last one):
+            //      warp w converts heads w, w+4, ...; a lane owns four consecutive dims
+            if (b != q_b || head != q_head) {
+                q_b = b;
+                q_head = head;
+                for (int h = gw; h < p.G; h += 4) {
+                    const uint2 raw = *reinterpret_cast<const uint2 *>(info + L::kQraw + h * 256 + lane * 8);
+                    const float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
+                                        bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
+                    const float am = warp_max(fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
+                    const float p2 = pow2_floor(am);
+                    const float f = pow2_recip(p2) * kStQFix;
+                    uint32_t lo_w = 0, hi_w = 0;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    // v = round(x * f), |v| < 16384, as the low 16 bits of 1.5 * 2^23 + v (two's complement)
-                    const int v = (int)(int16_t)(__float_as_uint(fmaf(x[i], f, 12582912.f)) & 0xFFFFu);
-                    const int hi = (v + 128) >> 8;            // v = 256 * hi + lo with lo in [-128, 127]
-                    lo_w |= ((uint32_t)v & 0xFFu) << (8 * i);
-                    hi_w |= ((uint32_t)hi & 0xFFu) << (8 * i);
+                    for (int i = 0; i < 4; ++i) {
+                        // v = round(x * f), |v| < 16384, as the low 16 bits of 1.5 * 2^23 + v (two's complement)
+                        const int v = (int)(int16_t)(__float_as_uint(fmaf(x[i], f, 12582912.f)) & 0xFFFFu);
+                        const int hi = (v + 128) >> 8;            // v = 256 * hi + lo with lo in [-128, 127]
+                        lo_w |= ((uint32_t)v & 0xFFu) << (8 * i);
+                        hi_w |= ((uint32_t)hi & 0xFFu) << (8 * i);
+                    }
+                    if (lane == 0) rowscale[h] = p2 * p.scale_log2e * (1.f / kStQFix);
+                    *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(h, 4 * lane)) = hi_w;
+                    *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(NH + h, 4 * lane)) = lo_w;
                 }
-                if (lane == 0) rowscale[h] = p2 * p.scale_log2e * (1.f / kStQFix);
-                *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(h, 4 * lane)) = hi_w;
-                *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(NH + h, 4 * lane)) = lo_w;
             }
             // this thread's two tokens
             float sk[2], lsv[2], rsv[2];
@@ -331,44 +452,12 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const float sv = valid[t] ? fmaxf(vs_s[tok], kMinScale) : 1.f;
                     sk[t] = valid[t] ? ks_s[tok] : 0.f;
                     lsv[t] = __log2f(sv);
-                    rsv[t] = valid[t] ? __frcp_rn(sv) : 0.f;
+                    rsv[t] = valid[t] ? st_rcp(sv) : 0.f;
                 }
             }
+            tc::mbar_arrive(bar_info_empty(islot));   // this thread has read everything it needs from the record
             tc::fence_proxy_async();
-            tc::named_barrier(bar_id, kStGroupThreads);
-
-            // ---- scores on the tensor cores; each K stage goes back to the producer when the MMAs have read it
-            if (gtid == 0) {
-                // every thread of the group has read the chunk record (scales, query rows, coordinates)
-                tc::mbar_arrive(bar_info_empty(islot));
-                constexpr uint32_t idesc = tc::instr_desc(2, 1, 1, false, false, 128, N);   // s32 <- s8 (K-major) x s8 (K-major)
-                int kst[2];
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t < n_tiles) {
-                        const int gi = tile0 + t;
-                        kst[t] = gi % S;
-                        wait(bar_full(kst[t]), (uint32_t)(gi / S) & 1u);
-                    }
-                }
-                tc::fence_after_sync();
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t < n_tiles) {
-                        const uint32_t k_addr = sbase + (uint32_t)kst[t] * kStTileBytes;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t a = tc::smem_desc(k_addr + j * 32, 16, 1024, tc::kSwizzle128B);
-                            const uint64_t bq = tc::smem_desc(grp_addr + L::kQop + j * 256, 128, 1024, tc::kSwizzleNone);
-                            tc::mma_i8(tm + t * N, a, bq, idesc, j > 0);
-                        }
-                    }
-                }
-                tc::commit(bar_mma_s(g));
-#pragma unroll
-                for (int t = 0; t < 2; ++t)
-                    if (t < n_tiles) tc::commit(bar_empty(kst[t]));
-            }
+            tc::mbar_arrive(bar_ready_s(g));          // the query operand is in place (128 arrivals start the score MMAs)
 
             wait(bar_mma_s(g), mph);
             __syncwarp();   // reconverge after the wait loop: the tensor-memory loads below are warp-aligned
@@ -402,11 +491,12 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     for (int h = 0; h < NH; ++h) s[t][h] = -INFINITY;
                 }
             }
+            // warp maxima by one integer reduction per head (the map float -> int below preserves the order)
 #pragma unroll
             for (int h = 0; h < NH; ++h) {
                 if (h < p.G) {
-                    const float m = warp_max(mloc[h]);
-                    if (lane == 0) red_m[h * 4 + gw] = m;
+                    const int m = __reduce_max_sync(0xffffffffu, st_ordered_int(mloc[h]));
+                    if (lane == 0) red_m[h * 4 + gw] = st_ordered_float(m);
                 }
             }
             tc::fence_before_sync();
@@ -422,7 +512,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         if (t < n_tiles) {
-                            const float e = exp2f(s[t][h] - M);
+                            const float e = st_exp2(s[t][h] - M);
                             lloc = fmaf(e, rsv[t], lloc);
                             const uint32_t bits = __float_as_uint(fmaf(e, kStPFix, 8388608.f));   // 2^23 + round(e * 65535)
                             unsigned char *pt = grp + L::kP + t * L::kPTileBytes;
@@ -430,43 +520,12 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                             pt[st_core_off(NH + h, gtid)] = (unsigned char)(bits & 0xFFu);
                         }
                     }
-                    const float l = warp_sum(lloc);
-                    if (lane == 0) red_l[h * 4 + gw] = l;
+                    lsum[h * kStGroupThreads + gtid] = lloc;
                 }
             }
             tc::fence_proxy_async();
-            tc::named_barrier(bar_id, kStGroupThreads);
+            tc::mbar_arrive(bar_ready_pv(g));         // P^T is in place (128 arrivals start the output MMAs)
 
-            // ---- O^T = V^T . P^T on the tensor cores; the V stages go back when the MMAs have read them
-            if (gtid == 0) {
-                constexpr uint32_t idesc = tc::instr_desc(2, 1, 0, true, false, 128, N);   // s32 <- s8 (MN-major) x u8 (K-major)
-                int vst[2];
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t < n_tiles) {
-                        const int gi = tile0 + n_tiles + t;
-                        vst[t] = gi % S;
-                        wait(bar_full(vst[t]), (uint32_t)(gi / S) & 1u);
-                    }
-                }
-                tc::fence_after_sync();
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t < n_tiles) {
-                        const uint32_t v_addr = sbase + (uint32_t)vst[t] * kStTileBytes;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t a = tc::smem_desc(v_addr + j * 4096, 1024, 1024, tc::kSwizzle128B);
-                            const uint64_t bp = tc::smem_desc(grp_addr + L::kP + t * L::kPTileBytes + j * 256, 128, 1024, tc::kSwizzleNone);
-                            tc::mma_i8(tm + 2 * N, a, bp, idesc, (t > 0) || (j > 0));
-                        }
-                    }
-                }
-                tc::commit(bar_mma_pv(g));
-#pragma unroll
-                for (int t = 0; t < 2; ++t)
-                    if (t < n_tiles) tc::commit(bar_empty(vst[t]));
-            }
             wait(bar_mma_pv(g), mph);
             __syncwarp();
             tc::fence_after_sync();
@@ -490,12 +549,26 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     }
                 }
             }
-            if (gtid < p.G) {
-                const size_t ps = ((size_t)b * p.Hq + h0 + gtid) * p.n_chunks + chunk;
-                const float4 mw = *reinterpret_cast<const float4 *>(red_m + gtid * 4);
-                const float4 lw = *reinterpret_cast<const float4 *>(red_l + gtid * 4);
-                p.part_ml[ps * 2] = fmaxf(fmaxf(mw.x, mw.y), fmaxf(mw.z, mw.w));
-                p.part_ml[ps * 2 + 1] = (lw.x + lw.y) + (lw.z + lw.w);
+            // ---- denominators: 128 / NH consecutive lanes add up one head's 128 shares (all of them were written
+            //      before the output MMAs started)
+            {
+                constexpr int kLanesPerHead = kStGroupThreads / NH;   // 16 or 8
+                const int h = gtid / kLanesPerHead, seg = gtid % kLanesPerHead;
+                const float4 *src = reinterpret_cast<const float4 *>(lsum + h * kStGroupThreads + seg * NH);
+                float l = 0.f;
+#pragma unroll
+                for (int i = 0; i < NH / 4; ++i) {
+                    const float4 v = src[i];
+                    l += (v.x + v.y) + (v.z + v.w);
+                }
+#pragma unroll
+                for (int o = kLanesPerHead / 2; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+                if (seg == 0 && h < p.G) {
+                    const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_chunks + chunk;
+                    const float4 mw = *reinterpret_cast<const float4 *>(red_m + h * 4);
+                    p.part_ml[ps * 2] = fmaxf(fmaxf(mw.x, mw.y), fmaxf(mw.z, mw.w));
+                    p.part_ml[ps * 2 + 1] = l;
+                }
             }
             // the next chunk's MMAs overwrite this group's tensor-memory columns: the loads above have retired
             tc::fence_before_sync();
