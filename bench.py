@@ -287,7 +287,7 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 mma, f32 accumulate",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8 (tcgen05 kind::i8 MMA, s32 accumulate; fp32 softmax)",
         "data": "synthetic",
         "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
                    "context": ctx + 1, "cache": "int8 codes + fp32 scale per (token, kv head), 128-token pages",
@@ -295,7 +295,7 @@ def run_ours(args, rank, world, local_rank):
                    "parallelism": f"dp{world} (independent sequences per GPU, no collective)"},
         "hbm_gbs_step_per_gpu": step_bytes / (ms_total / args.steps * 1e-3) / 1e9,
         "pct_of_8tbs_step": 100.0 * step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / 8000.0,
-        "roofline": {"bound": "hbm", "kernel": "slim_decode_split_kernel", "achieved": achieved, "peak": hbm_peak,
+        "roofline": {"bound": "hbm", "kernel": "slim_decode_stream_kernel", "achieved": achieved, "peak": hbm_peak,
                      "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_8tbs": achieved / 8000.0, "bytes_per_launch": split_bytes,
                      "avg_launch_ms": split_avg_ms, "min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},

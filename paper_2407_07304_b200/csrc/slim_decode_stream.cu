@@ -168,21 +168,51 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     }
     if (warp == 8) {
         tc::tmem_alloc(smem_u32(tmem_slot), kStTmemCols);
-        // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order
-        long long chunks_all = 0;
-        for (int base = 0; base < B; base += 32) {
+        // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order.  The work is cut
+        //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.
+        const int len_first = (lane < B) ? st_clamped_len(p, lane) : 0;   // the first 32 sequences stay in registers
+        auto seq_len = [&](int base) {
             const int b = base + lane;
-            const int nc = (b < B) ? (st_clamped_len(p, b) + kStChunk - 1) / kStChunk : 0;
-            chunks_all += __reduce_add_sync(0xffffffffu, nc);
-        }
-        const long long total = chunks_all * p.Hkv;
-        const long long i0 = total * blockIdx.x / gridDim.x, i1 = total * (blockIdx.x + 1) / gridDim.x;
+            return (base == 0) ? len_first : ((b < B) ? st_clamped_len(p, b) : 0);
+        };
+        long long tiles_all = 0;
+        for (int base = 0; base < B; base += 32)
+            tiles_all += __reduce_add_sync(0xffffffffu, (seq_len(base) + kStTile - 1) / kStTile);
+        const long long total_tiles = tiles_all * p.Hkv;
+        // number of chunks that start before tile index x (x <= total_tiles), over all (sequence, kv head) runs in order
+        auto chunks_before = [&](long long x) {
+            long long tiles_pre = 0, chunks_pre = 0;
+            for (int base = 0; base < B; base += 32) {
+                const int len = seq_len(base);
+                const int nt = (len + kStTile - 1) / kStTile, nc = (len + kStChunk - 1) / kStChunk;
+                int it = nt, ic = nc;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int vt = __shfl_up_sync(0xffffffffu, it, o), vc = __shfl_up_sync(0xffffffffu, ic, o);
+                    if (lane >= o) it += vt, ic += vc;
+                }
+                const unsigned hit = __ballot_sync(0xffffffffu, (tiles_pre + it) * p.Hkv > x);
+                if (hit != 0u) {
+                    const int l = __ffs(hit) - 1;
+                    const int nt_l = __shfl_sync(0xffffffffu, nt, l), nc_l = __shfl_sync(0xffffffffu, nc, l);
+                    const long long tb = tiles_pre + __shfl_sync(0xffffffffu, it, l) - nt_l;
+                    const long long cb = chunks_pre + __shfl_sync(0xffffffffu, ic, l) - nc_l;
+                    const long long r = x - tb * p.Hkv;              // < Hkv * nt_l
+                    const int head = (int)(r / nt_l), d = (int)(r % nt_l);
+                    return cb * p.Hkv + (long long)head * nc_l + min(nc_l, (d + 1) / 2);
+                }
+                tiles_pre += __shfl_sync(0xffffffffu, it, 31);
+                chunks_pre += __shfl_sync(0xffffffffu, ic, 31);
+            }
+            return chunks_pre * p.Hkv;
+        };
+        const long long i0 = chunks_before(total_tiles * blockIdx.x / gridDim.x);
+        const long long i1 = chunks_before(total_tiles * (blockIdx.x + 1) / gridDim.x);
         int b0 = 0, head0 = 0, chunk0 = 0;
         if (i1 > i0) {
             long long prefix = 0;   // chunks of the sequences before `base`
             for (int base = 0; base < B; base += 32) {
-                const int b = base + lane;
-                const int nc = (b < B) ? (st_clamped_len(p, b) + kStChunk - 1) / kStChunk : 0;
+                const int nc = (seq_len(base) + kStChunk - 1) / kStChunk;
                 int incl = nc;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
