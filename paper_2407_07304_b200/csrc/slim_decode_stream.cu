@@ -6,17 +6,18 @@
 //
 //  * One thread block per SM.  The work - every 256-token chunk of every (sequence, kv head) - is cut
 //    into one contiguous range per block.  A chunk is the unit of a partial result (m, l, O[128]).
-//  * Warp 8 is the producer: one thread walks the block's chunks and asks the TMA engine for each
+//  * One warp is the producer: one thread walks the block's chunks and asks the TMA engine for each
 //    chunk's INT8 K tiles and V tiles into a ring of 16 KB tile stages (128-byte swizzled, completion
 //    counted on mbarriers) and for its scales and query rows into a small ring of chunk records.  A
 //    stage goes back to the producer the moment the tensor cores have read it (the MMA completion
 //    itself arrives on the stage's mbarrier), so K tiles are held only until the scores are out and
 //    most of the ring is in flight at any time.  A ragged last tile is fetched in 16-row boxes so
 //    that no byte beyond the chunk's tokens (rounded up to 16) is read.
-//  * Warps 9 and 10 each hold one MMA-issuing thread, one per consumer group: it waits for the chunk's
+//  * One more warp per consumer group holds that group's MMA-issuing thread: it waits for the chunk's
 //    tiles and for the group's operands, issues the tcgen05.mma instructions and commits their
 //    completion to the group's mbarrier and to the stages' "empty" mbarriers.
-//  * Warps 0-3 and 4-7 are two consumer groups that take chunks alternately.  For its chunk a group
+//  * Three consumer groups of four warps (two when a kv head serves more than eight query heads) take
+//    chunks in turn.  For its chunk a group
 //      - builds the query operand: a 14-bit fixed-point copy of the G = Hq/Hkv query rows of the kv
 //        head, two signed bytes per value (columns [high bytes | low bytes]);
 //      - S^T[token][head] = K_codes . Q^T by tcgen05.mma kind::i8: the INT8 codes are the operand as
@@ -26,7 +27,7 @@
 //      - O^T[dim][head] = V_codes^T . P^T, again kind::i8, V read MN-major straight from its
 //        token-major rows, P as 16-bit fixed point in two unsigned bytes;
 //      - recombines 256 * high + low exactly in int32 and writes the partial.
-//    While one group computes, the other group's chunk and the next chunk are in flight.
+//    While one group computes, the other groups' chunks and the next chunks are in flight.
 //
 // The V scale is folded into the softmax weight (s'_j = s_j + log2 sv_j, P_j = 2^(s'_j - max s'),
 // o = sum P_j c_j / sum P_j / sv_j), so P <= 1 is normalised by the chunk's largest contribution.
@@ -40,33 +41,33 @@
 
 namespace slim {
 
-constexpr int kStGroups = 2;
 constexpr int kStGroupThreads = 128;
-constexpr int kStThreads = kStGroups * kStGroupThreads + 32 + kStGroups * 32;   // consumer groups + producer warp + one MMA-issue warp per group
-constexpr int kStInfoSlots = 4;                                 // chunk records in flight
 constexpr int kStTile = 128;                                    // tokens per MMA tile (= one page)
 constexpr int kStChunk = 2 * kStTile;                           // tokens per chunk / partial
 constexpr int kStTailBox = 16;                                  // rows per TMA box of a ragged tile
 constexpr uint32_t kStTileBytes = kStTile * kHeadDim;           // 16 KB
 constexpr float kStQFix = 8192.f;      // |q / pow2| < 2  ->  |v| < 16384, high byte in [-64, 64]
 constexpr float kStPFix = 65535.f;
-constexpr uint32_t kStTmemCols = 256;  // 128 per group: S of two tiles + O
 
 static_assert(kStChunk == 256, "partials are indexed by 256-token chunks (decode_workspace_bytes, merge kernel)");
 
 template <int NH>
 struct StSmem {
     static constexpr int N = 2 * NH;                        // MMA columns: [hi bytes of NH heads | lo bytes]
-    static constexpr int kStages = (NH <= 8) ? 11 : 10;     // tile stages of the ring
+    static constexpr int kGroups = (NH <= 8) ? 3 : 2;       // consumer groups (chunks in process at a time)
+    static constexpr int kThreads = kGroups * kStGroupThreads + 64 + kGroups * 32;   // groups + two producer warps + one MMA-issue warp per group
+    static constexpr int kProducerWarp = kGroups * 4;
+    static constexpr int kInfoSlots = 2 * kGroups;          // chunk records in flight
+    static constexpr uint32_t kTmemCols = (kGroups <= 2) ? 256 : 512;   // 128 per group: S of two tiles + O
+    static constexpr int kStages = 10;                      // tile stages of the ring
     // chunk record: both scale vectors, the kv head's query rows, the chunk's coordinates
-    static constexpr uint32_t kKs = 0;                      // 256 K scales
-    static constexpr uint32_t kVs = 1024;                   // 256 V scales
+    static constexpr uint32_t kScales = 0;                  // per tile: 128 K scales, then 128 V scales
     static constexpr uint32_t kQraw = 2048;                 // bf16 [G][128]
     static constexpr uint32_t kMeta = kQraw + NH * 256;     // int[5]: sequence, kv head, chunk, valid tokens, first tile index
     static constexpr uint32_t kInfoBytes = (kMeta + 32 + 127) / 128 * 128;
     static constexpr uint32_t kInfo0 = kStages * kStTileBytes;
     // per consumer group
-    static constexpr uint32_t kGroup0 = kInfo0 + kStInfoSlots * kInfoBytes;
+    static constexpr uint32_t kGroup0 = kInfo0 + kInfoSlots * kInfoBytes;
     static constexpr uint32_t kPTileBytes = N * 128;        // a P^T tile, core-matrix layout
     static constexpr uint32_t kP = 0;                       // two P^T tiles
     static constexpr uint32_t kQop = 2 * kPTileBytes;       // query operand: N rows x 128 bytes, core-matrix layout
@@ -75,8 +76,8 @@ struct StSmem {
     static constexpr uint32_t kGroupBytes = (kRed + 5 * NH * 4 + 127) / 128 * 128;
     // block-wide: mbarriers full[kStages], empty[kStages], info full[4], info empty[4],
     //             operands ready for S[2], for PV[2], S done[2], PV done[2]
-    static constexpr uint32_t kBar = kGroup0 + kStGroups * kGroupBytes;
-    static constexpr int kNumBars = 2 * kStages + 2 * kStInfoSlots + 4 * kStGroups;
+    static constexpr uint32_t kBar = kGroup0 + kGroups * kGroupBytes;
+    static constexpr int kNumBars = 2 * kStages + 2 * kInfoSlots + 4 * kGroups;
     static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
     static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[4]: chunks of this block, first sequence / head / chunk
     static constexpr uint32_t kFail = kRange + 16;
@@ -124,13 +125,15 @@ __device__ __forceinline__ int st_clamped_len(const DecodeParams &p, int b)
 }
 
 template <int NH>
-__global__ void __launch_bounds__(kStThreads, 1)
+__global__ void __launch_bounds__(StSmem<NH>::kThreads, 1)
 slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __grid_constant__ CUtensorMap map_tail,
                           const DecodeParams p, const int B)
 {
     using L = StSmem<NH>;
     constexpr int N = L::N;
     constexpr int S = L::kStages;
+    constexpr int kStGroups = L::kGroups, kStInfoSlots = L::kInfoSlots;
+    constexpr int kPW = L::kProducerWarp;
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t sbase = smem_u32(smem);
@@ -166,8 +169,8 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         tc::mbar_init_fence();
         *fail = 0;
     }
-    if (warp == 8) {
-        tc::tmem_alloc(smem_u32(tmem_slot), kStTmemCols);
+    if (warp == kPW) {
+        tc::tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
         // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order.  The work is cut
         //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.
         const int len_first = (lane < B) ? st_clamped_len(p, lane) : 0;   // the first 32 sequences stay in registers
@@ -239,7 +242,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             range[2] = head0;
             range[3] = chunk0;
         }
-    } else if (warp < 8) {
+    } else if (warp < kPW) {
         // rows of the query operand that belong to no head stay zero for the whole launch
         const int g = warp >> 2, gtid = tid & 127;
         unsigned char *qop = smem + L::kGroup0 + g * L::kGroupBytes + L::kQop;
@@ -260,8 +263,12 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     };
     int tiles_issued = 0;   // producer thread: tile stages armed so far (ring position)
 
-    if (warp == 8) {
-        // =========================================================== producer (one thread)
+    if (warp == kPW || warp == kPW + 1) {
+        // =========================================================== producers (one thread each)
+        // warp kPW walks the block's chunks and asks for their K and V tiles; warp kPW + 1 walks the same
+        // list and asks for the chunk records (coordinates, scales, query rows).  Two threads because
+        // the rate at which one thread can hand requests to the copy engine would otherwise limit the stream.
+        const bool tile_role = warp == kPW;
         if (lane == 0 && cnt > 0) {
             int b = range[1], head = range[2], chunk = range[3];
             int len = st_clamped_len(p, b);
@@ -277,8 +284,6 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             int stage = 0;
             uint32_t stage_ph = 0;   // parity of the stage's current use
             for (int n = 0; n < cnt; ++n) {
-                const int islot = n % kStInfoSlots;
-                const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
                 const int cb = b, chead = head, cchunk = chunk;
                 const int n_tok = min(kStChunk, len - chunk * kStChunk);
                 const int2 cpg = pg;
@@ -305,53 +310,61 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const int rows = max(0, min(kStTile, n_tok - t * kStTile));
                     rows16[t] = (rows + kStTailBox - 1) / kStTailBox * kStTailBox;
                 }
-                // ---- the chunk record: coordinates, both scale vectors, the query rows
-                wait(bar_info_empty(islot), iph ^ 1u);
-                unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
-                const uint32_t info_addr = sbase + L::kInfo0 + islot * L::kInfoBytes;
-                int *meta = reinterpret_cast<int *>(info + L::kMeta);
-                meta[0] = cb, meta[1] = chead, meta[2] = cchunk, meta[3] = n_tok, meta[4] = tiles_issued;
-                const uint32_t q_bytes = (uint32_t)p.G * kHeadDim * 2u;
-                tc::mbar_arrive_expect_tx(bar_info_full(islot), 2u * (uint32_t)(rows16[0] + rows16[1]) * 4u + q_bytes);
+                const int n_tiles = rows16[1] > 0 ? 2 : 1;
+                if (!tile_role) {
+                    // ---- the chunk record: coordinates, the scales of its tiles (K and V scales of a page and head
+                    //      are adjacent: one 1 KB copy per tile), and the query rows unless the group that takes
+                    //      this chunk still holds them from its previous chunk (same sequence and kv head)
+                    const int islot = n % kStInfoSlots;
+                    const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
+                    wait(bar_info_empty(islot), iph ^ 1u);
+                    unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
+                    const uint32_t info_addr = sbase + L::kInfo0 + islot * L::kInfoBytes;
+                    int *meta = reinterpret_cast<int *>(info + L::kMeta);
+                    meta[0] = cb, meta[1] = chead, meta[2] = cchunk, meta[3] = n_tok, meta[4] = tiles_issued;
+                    const bool need_q = !(n >= kStGroups && cchunk >= kStGroups);
+                    const uint32_t q_bytes = need_q ? (uint32_t)p.G * kHeadDim * 2u : 0u;
+                    tc::mbar_arrive_expect_tx(bar_info_full(islot), (uint32_t)n_tiles * 1024u + q_bytes);
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (rows16[t] == 0) continue;
-                    tc::bulk_load(info_addr + L::kKs + t * 512, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
-                                  (uint32_t)rows16[t] * 4u, bar_info_full(islot));
-                    tc::bulk_load(info_addr + L::kVs + t * 512, p.scales + scale_block_offset(page[t], chead, 1, p.Hkv),
-                                  (uint32_t)rows16[t] * 4u, bar_info_full(islot));
-                }
-                tc::bulk_load(info_addr + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes,
-                              bar_info_full(islot));
-                // ---- the chunk's tiles, in the order the consumers need them: K tiles, then V tiles
+                    for (int t = 0; t < 2; ++t)
+                        if (t < n_tiles)
+                            tc::bulk_load(info_addr + L::kScales + t * 1024, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
+                                          1024u, bar_info_full(islot));
+                    if (need_q)
+                        tc::bulk_load(info_addr + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes,
+                                      bar_info_full(islot));
+                    tiles_issued += 2 * n_tiles;
+                } else {
+                    // ---- the chunk's tiles, in the order the consumers need them: K tiles, then V tiles
 #pragma unroll
-                for (int kv = 0; kv < 2; ++kv) {
+                    for (int kv = 0; kv < 2; ++kv) {
 #pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        if (rows16[t] == 0) continue;
-                        wait(bar_empty(stage), stage_ph ^ 1u);
-                        const uint32_t full = bar_full(stage);
-                        tc::mbar_arrive_expect_tx(full, (uint32_t)rows16[t] * kHeadDim);
-                        const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
-                        const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
-                        if (rows16[t] == kStTile) {
-                            tc::tma_load_2d(dst, &map_tile, 0, row0, full);
-                        } else {
-                            for (int r = 0; r < rows16[t]; r += kStTailBox)
-                                tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
-                        }
-                        ++tiles_issued;
-                        if (++stage == S) {
-                            stage = 0;
-                            stage_ph ^= 1u;
+                        for (int t = 0; t < 2; ++t) {
+                            if (rows16[t] == 0) continue;
+                            wait(bar_empty(stage), stage_ph ^ 1u);
+                            const uint32_t full = bar_full(stage);
+                            tc::mbar_arrive_expect_tx(full, (uint32_t)rows16[t] * kHeadDim);
+                            const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
+                            const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
+                            if (rows16[t] == kStTile) {
+                                tc::tma_load_2d(dst, &map_tile, 0, row0, full);
+                            } else {
+                                for (int r = 0; r < rows16[t]; r += kStTailBox)
+                                    tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
+                            }
+                            ++tiles_issued;
+                            if (++stage == S) {
+                                stage = 0;
+                                stage_ph ^= 1u;
+                            }
                         }
                     }
                 }
             }
         }
-    } else if (warp >= 9) {
+    } else if (warp > kPW + 1) {
         // =========================================================== MMA issue for group g (one thread)
-        const int g = warp - 9;
+        const int g = warp - kPW - 2;
         if (lane == 0) {
             const uint32_t grp_addr = sbase + L::kGroup0 + g * L::kGroupBytes;
             const uint32_t tm = tmem + (uint32_t)g * 128u;
@@ -473,14 +486,13 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             float sk[2], lsv[2], rsv[2];
             bool valid[2];
             {
-                const float *ks_s = reinterpret_cast<const float *>(info + L::kKs);
-                const float *vs_s = reinterpret_cast<const float *>(info + L::kVs);
+                const float *sc = reinterpret_cast<const float *>(info + L::kScales);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     const int tok = t * kStTile + gtid;
                     valid[t] = tok < n_tok;
-                    const float sv = valid[t] ? fmaxf(vs_s[tok], kMinScale) : 1.f;
-                    sk[t] = valid[t] ? ks_s[tok] : 0.f;
+                    const float sv = valid[t] ? fmaxf(sc[t * 256 + 128 + gtid], kMinScale) : 1.f;
+                    sk[t] = valid[t] ? sc[t * 256 + gtid] : 0.f;
                     lsv[t] = __log2f(sv);
                     rsv[t] = valid[t] ? st_rcp(sv) : 0.f;
                 }
@@ -607,7 +619,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 
     tc::fence_before_sync();
     __syncthreads();
-    if (warp == 8) {
+    if (warp == kPW) {
         if (lane == 0 && *fail != 0) {
             // a wait ran out somewhere: give the copies still in flight a bounded chance to land before the block exits
             for (int gi = max(0, tiles_issued - S); gi < tiles_issued; ++gi)
@@ -618,7 +630,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         }
         __syncwarp();
         tc::fence_after_sync();
-        tc::tmem_dealloc(tmem, kStTmemCols);
+        tc::tmem_dealloc(tmem, L::kTmemCols);
     }
 }
 
@@ -637,11 +649,11 @@ int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int
     if (p.G <= 8) {
         constexpr int bytes = (int)StSmem<8>::kBytes;
         SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-        slim_decode_stream_kernel<8><<<grid, kStThreads, bytes, stream>>>(map_tile, map_tail, p, B);
+        slim_decode_stream_kernel<8><<<grid, StSmem<8>::kThreads, bytes, stream>>>(map_tile, map_tail, p, B);
     } else {
         constexpr int bytes = (int)StSmem<16>::kBytes;
         SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-        slim_decode_stream_kernel<16><<<grid, kStThreads, bytes, stream>>>(map_tile, map_tail, p, B);
+        slim_decode_stream_kernel<16><<<grid, StSmem<16>::kThreads, bytes, stream>>>(map_tile, map_tail, p, B);
     }
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
