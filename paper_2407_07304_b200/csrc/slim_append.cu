@@ -29,6 +29,7 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
                    const int32_t *__restrict__ cu_new, const int32_t *__restrict__ start_pos,
                    int Hkv, int max_pages_per_seq, int num_pages)
 {
+    pdl_launch_dependents();   // a decode kernel queued behind this one may run its set-up meanwhile
     const int b = blockIdx.y;
     const int kv = blockIdx.z;
     const int hw = threadIdx.x >> 4, l = threadIdx.x & 15;

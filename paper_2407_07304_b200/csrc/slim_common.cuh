@@ -31,6 +31,30 @@ __host__ __device__ inline size_t scale_block_offset(int page, int head, int kv,
     return ((size_t)((size_t)page * Hkv + head) * 2 + kv) * (size_t)kPageTokens;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with launch_pdl() may start while the kernel before it in the stream is still
+// running (once every block of that kernel has called pdl_launch_dependents() or exited); it must call
+// pdl_wait() before it touches anything the earlier kernel writes.  pdl_wait() returns when the
+// earlier kernel has completed and its writes are visible; without an earlier kernel it returns at once.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---------------------------------------------------------------- cp.async (16-byte global -> shared)
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {

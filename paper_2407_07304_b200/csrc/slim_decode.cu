@@ -423,6 +423,7 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
 {
     const int row = blockIdx.x * 4 + (threadIdx.x >> 5);   // b * Hq + h
     const int lane = threadIdx.x & 31;
+    pdl_wait();   // the split pass before this kernel must have finished writing the partials
     if (row >= B * Hq) return;
     const int b = row / Hq;
     const int len = kv_len[b];
@@ -517,10 +518,8 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
     int C;
     const DecodeParams p = make_params(c, nullptr, kv_len, B, max_kv, Hq, 1.f, const_cast<void *>(workspace), C);
     const int rows = B * Hq;
-    slim_decode_merge_kernel<<<(rows + 3) / 4, 128, 0, stream>>>(p.part_o, p.part_ml, kv_len,
-                                                                 static_cast<__nv_bfloat16 *>(out), B, Hq,
-                                                                 p.n_chunks, C);
-    SLIM_CUDA_TRY(cudaGetLastError());
+    SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel, dim3((rows + 3) / 4), dim3(128), 0, stream, (const float *)p.part_o,
+                             (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
     return SLIM_OK;
 }
 

@@ -150,6 +150,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     int *range = reinterpret_cast<int *>(smem + L::kRange);
     volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
 
+    pdl_launch_dependents();   // the merge kernel queued behind this one may be scheduled; it waits for our completion
     if (tid == 0) {
         for (int i = 0; i < S; ++i) {
             tc::mbar_init(bar_full(i), 1);
@@ -171,6 +172,9 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     }
     if (warp == kPW) {
         tc::tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
+        // Up to here the block may run beside the kernel before it in the stream (the same step's
+        // slim_kv_append); from here on it reads what earlier kernels may have written.
+        pdl_wait();
         // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order.  The work is cut
         //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.
         const int len_first = (lane < B) ? st_clamped_len(p, lane) : 0;   // the first 32 sequences stay in registers
@@ -270,6 +274,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         // the rate at which one thread can hand requests to the copy engine would otherwise limit the stream.
         const bool tile_role = warp == kPW;
         if (lane == 0 && cnt > 0) {
+            pdl_wait();   // (returns at once: the earlier kernel was already waited for before the lengths were read)
             int b = range[1], head = range[2], chunk = range[3];
             int len = st_clamped_len(p, b);
             int nc = (len + kStChunk - 1) / kStChunk;
@@ -649,11 +654,11 @@ int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int
     if (p.G <= 8) {
         constexpr int bytes = (int)StSmem<8>::kBytes;
         SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-        slim_decode_stream_kernel<8><<<grid, StSmem<8>::kThreads, bytes, stream>>>(map_tile, map_tail, p, B);
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<8>, dim3(grid), dim3(StSmem<8>::kThreads), bytes, stream, map_tile, map_tail, p, B));
     } else {
         constexpr int bytes = (int)StSmem<16>::kBytes;
         SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
-        slim_decode_stream_kernel<16><<<grid, StSmem<16>::kThreads, bytes, stream>>>(map_tile, map_tail, p, B);
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<16>, dim3(grid), dim3(StSmem<16>::kThreads), bytes, stream, map_tile, map_tail, p, B));
     }
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
