@@ -260,7 +260,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     const int cnt = range[0];
     bool ok = true;
     auto wait = [&](uint32_t mbar, uint32_t parity) {
-        if (!tc::mbar_wait(mbar, parity, (ok && *fail == 0) ? (1u << 18) : 1u)) {
+        if (!tc::mbar_wait(mbar, parity, ok ? (1u << 18) : 1u, fail)) {
             ok = false;
             *fail = 1;
         }
@@ -375,6 +375,11 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             const uint32_t tm = tmem + (uint32_t)g * 128u;
             constexpr uint32_t idesc_s = tc::instr_desc(2, 1, 1, false, false, 128, N);    // s32 <- s8 (K-major) x s8 (K-major)
             constexpr uint32_t idesc_pv = tc::instr_desc(2, 1, 0, true, false, 128, N);    // s32 <- s8 (MN-major) x u8 (K-major)
+            // operand descriptors are built once; an MMA step only adds a constant to the address field
+            const uint64_t dk0 = tc::smem_desc(sbase, 16, 1024, tc::kSwizzle128B);         // a K tile in stage 0
+            const uint64_t dv0 = tc::smem_desc(sbase, 1024, 1024, tc::kSwizzle128B);       // a V tile in stage 0 (MN-major)
+            const uint64_t dq = tc::smem_desc(grp_addr + L::kQop, 128, 1024, tc::kSwizzleNone);
+            const uint64_t dp = tc::smem_desc(grp_addr + L::kP, 128, 1024, tc::kSwizzleNone);
             for (int n = g; n < cnt; n += kStGroups) {
                 const int islot = n % kStInfoSlots;
                 const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
@@ -401,13 +406,10 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (t < n_tiles) {
-                        const uint32_t k_addr = sbase + (uint32_t)st[t] * kStTileBytes;
+                        const uint64_t a = dk0 + (uint64_t)((uint32_t)st[t] * (kStTileBytes >> 4));
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t a = tc::smem_desc(k_addr + j * 32, 16, 1024, tc::kSwizzle128B);
-                            const uint64_t bq = tc::smem_desc(grp_addr + L::kQop + j * 256, 128, 1024, tc::kSwizzleNone);
-                            tc::mma_i8(tm + t * N, a, bq, idesc_s, j > 0);
-                        }
+                        for (int j = 0; j < 4; ++j)   // 32 dims per step: 32 bytes inside the swizzle span; 256 bytes of the query operand
+                            tc::mma_i8(tm + t * N, a + (uint64_t)(j * 2), dq + (uint64_t)(j * 16), idesc_s, j > 0);
                     }
                 }
                 tc::commit(bar_mma_s(g));
@@ -423,13 +425,11 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (t < n_tiles) {
-                        const uint32_t v_addr = sbase + (uint32_t)st[n_tiles + t] * kStTileBytes;
+                        const uint64_t a = dv0 + (uint64_t)((uint32_t)st[n_tiles + t] * (kStTileBytes >> 4));
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t a = tc::smem_desc(v_addr + j * 4096, 1024, 1024, tc::kSwizzle128B);
-                            const uint64_t bp = tc::smem_desc(grp_addr + L::kP + t * L::kPTileBytes + j * 256, 128, 1024, tc::kSwizzleNone);
-                            tc::mma_i8(tm + 2 * N, a, bp, idesc_pv, (t > 0) || (j > 0));
-                        }
+                        for (int j = 0; j < 4; ++j)   // 32 tokens per step: 4 KB down the V tile; 256 bytes of the P^T tile
+                            tc::mma_i8(tm + 2 * N, a + (uint64_t)(j * 256), dp + (uint64_t)((t * L::kPTileBytes + j * 256) >> 4), idesc_pv,
+                                       (t > 0) || (j > 0));
                     }
                 }
                 tc::commit(bar_mma_pv(g));

@@ -12,12 +12,14 @@
 //   warps 8-11  dequantise in registers (the hybrid-dtype step of Section 2.2): INT8 codes -> fp16
 //               code * scale / 2^e, written in the swizzled layout the tensor cores read (one K and
 //               one V operand buffer; a buffer is refilled as soon as the MMAs that read it are done)
-//   warp 13     one thread issues tcgen05.mma in the order  P0.V(j), Q0.K(j+1)^T, P1.V(j), Q1.K(j+1)^T:
+//   warps 13,14 one MMA-issuing thread per query tile, each in the order  P_t.V(j), Q_t.K(j+1)^T:
 //               S_t = Q_t . K^T (both operands in shared memory), O_t += P_t . V (P read from tensor
-//               memory), fp32 accumulators in tensor memory
-//   warps 0-3   softmax of Q0, warps 4-7 softmax of Q1; thread = query row.  Two passes over the score row
-//               in 32-column pieces (tcgen05.ld): row maximum, then exp2 -> fp16 P back to tensor memory
-//               and the running sum.  O is rescaled only when the maximum grows by more than 2^8.
+//               memory), fp32 accumulators in tensor memory.  Two threads so that neither tile waits for
+//               the other one's softmax.
+//   warps 0-3   softmax of Q0, warps 4-7 softmax of Q1; thread = query row.  The whole 128-column score row is
+//               read into registers with one tcgen05.ld round trip (the softmax warps take registers from the
+//               other warp groups: setmaxnreg), then row maximum, exp2 -> fp16 P back to tensor memory and the
+//               running sum.  O is rescaled only when the maximum grows by more than 2^8.
 //
 // Scale bookkeeping: K^ = code * sk / kexp(j) with kexp(j) the power of two below the tile's largest K
 // scale, so s = acc * (kexp * row_scale); V^ = code * sv / vnorm with vnorm the power of two below the
@@ -31,7 +33,7 @@
 
 namespace slim {
 
-constexpr int kPfThreads = 448;
+constexpr int kPfThreads = 512;   // four warp groups: softmax 0, softmax 1, dequantisers, {loader, two MMA threads, one idle warp}
 constexpr int kPfBM = 128, kPfBN = 128;
 constexpr int kPfRows = 2 * kPfBM;             // query rows per block
 constexpr int kPfRawStages = 5;
@@ -72,6 +74,12 @@ __device__ __forceinline__ float pf_exp2(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ float pf_max3(float a, float b, float c)
+{
+    float m;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
 }
 __device__ __forceinline__ uint32_t pf_hsub2(uint32_t a, uint32_t b)
 {
@@ -124,9 +132,9 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             tc::mbar_init(bar(pfl::RAW_EMPTY, i), 128);
         }
         tc::mbar_init(bar(pfl::KF_FULL, 0), 128);
-        tc::mbar_init(bar(pfl::KF_EMPTY, 0), 1);
+        tc::mbar_init(bar(pfl::KF_EMPTY, 0), 2);   // both MMA threads are done with the K tile
         tc::mbar_init(bar(pfl::VF_FULL, 0), 128);
-        tc::mbar_init(bar(pfl::VF_EMPTY, 0), 1);
+        tc::mbar_init(bar(pfl::VF_EMPTY, 0), 2);
         for (int t = 0; t < 2; ++t) {
             tc::mbar_init(bar(pfl::S_FULL, t), 1);
             tc::mbar_init(bar(pfl::P_FULL, t), 128);
@@ -143,12 +151,22 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     const uint32_t tmem = *tmem_slot;
     bool ok = true;
     auto wait = [&](uint32_t mbar, uint32_t parity) {
-        if (!tc::mbar_wait(mbar, parity, (ok && *fail == 0) ? (1u << 18) : 1u)) {
+        if (!tc::mbar_wait(mbar, parity, ok ? (1u << 18) : 1u, fail)) {
             ok = false;
             *fail = 1;
         }
     };
     int raw_issued = 0;   // loader thread: raw tiles requested so far
+
+    // Registers move from the warp groups that need few to the softmax groups, which hold a whole 128-column
+    // score row (every warp of a group executes the same setmaxnreg; 2 * 192 + 72 + 56 = 4 * 128 per lane).
+    if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 192;\n");
+    } else if (warp < 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;\n");
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;\n");
+    }
 
     if (warp < 8) {
         // =========================================================== softmax of query tile t: thread = query row
@@ -205,21 +223,33 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             const float c = fmaxf(rs * misc_f[j & 1], 1e-37f);   // row scale * kexp of this key tile (> 0)
             const int key0 = j * kPfBN;
             const bool diag = key0 + kPfBN - 1 > last_key;       // some of this tile's keys are masked for this row
-            // ---- pass 1: row maximum of the raw accumulators (c > 0, so the maximum commutes with the scaling)
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t v[32];
-                tc::tmem_ld32(tS + c4 * 32, v);
+            // ---- the whole score row into registers with one round trip to tensor memory, then its maximum
+            //      (c > 0, so the maximum of the raw accumulators commutes with the scaling)
+            uint32_t v[128];
+            {
+                uint32_t(&v0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&v[0]);
+                uint32_t(&v1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&v[32]);
+                uint32_t(&v2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&v[64]);
+                uint32_t(&v3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&v[96]);
+                tc::tmem_ld32(tS, v0);
+                tc::tmem_ld32(tS + 32, v1);
+                tc::tmem_ld32(tS + 64, v2);
+                tc::tmem_ld32(tS + 96, v3);
                 tc::tmem_ld_wait();
-                if (diag) {
+            }
+            float mx = -INFINITY;
+            if (diag) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (key0 + c4 * 32 + i <= last_key) mx = fmaxf(mx, __uint_as_float(v[i]));
-                } else {
+                for (int i = 0; i < 128; ++i)
+                    if (key0 + i <= last_key) mx = fmaxf(mx, __uint_as_float(v[i]));
+            } else {
+                float mx2 = -INFINITY;   // two chains
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(v[i]), __uint_as_float(v[i + 1])));
+                for (int i = 0; i < 128; i += 4) {
+                    mx = pf_max3(mx, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                    mx2 = pf_max3(mx2, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
                 }
+                mx = fmaxf(mx, mx2);
             }
             const float mt = (mx == -INFINITY) ? -INFINITY : mx * c;
             // the reference maximum only moves when the tile's exceeds it by more than the threshold
@@ -229,41 +259,39 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 wait(bar(pfl::O_DONE, t), (uint32_t)(j - 1) & 1u);      // P.V of the previous tile is complete
                 __syncwarp();
                 tc::fence_after_sync();
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint32_t v[32];
-                    tc::tmem_ld32(tO + c4 * 32, v);
+#pragma unroll 1
+                for (int k = 0; k < 8; ++k) {
+                    uint32_t v[16];
+                    tc::tmem_ld16(tO + k * 16, v);
                     tc::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                    tc::tmem_st32(tO + c4 * 32, v);
+                    for (int i = 0; i < 16; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                    tc::tmem_st16(tO + k * 16, v);
                 }
                 tc::tmem_st_wait();
                 l_run *= alpha;
             }
             if (grow) m_run = mt;
             const float bias = (m_run == -INFINITY) ? 0.f : -m_run;
-            // ---- pass 2: P = 2^(s - m) as fp16 into the first 64 columns of the score buffer, running sum
-            float rowsum = 0.f;
+            // ---- P = 2^(s - m) as fp16 pairs, packed in place, into the first 64 columns of the score buffer
+            float rowsum = 0.f, rowsum2 = 0.f;
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t v[32];
-                tc::tmem_ld32(tS + c4 * 32, v);
-                tc::tmem_ld_wait();
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float e0 = pf_exp2(fmaf(__uint_as_float(v[2 * i]), c, bias));
-                    float e1 = pf_exp2(fmaf(__uint_as_float(v[2 * i + 1]), c, bias));
-                    if (diag) {
-                        if (key0 + c4 * 32 + 2 * i > last_key) e0 = 0.f;
-                        if (key0 + c4 * 32 + 2 * i + 1 > last_key) e1 = 0.f;
-                    }
-                    rowsum += e0 + e1;
-                    pk[i] = pack_half2(e0, e1);
+            for (int i = 0; i < 64; ++i) {
+                float e0 = pf_exp2(fmaf(__uint_as_float(v[2 * i]), c, bias));
+                float e1 = pf_exp2(fmaf(__uint_as_float(v[2 * i + 1]), c, bias));
+                if (diag) {
+                    if (key0 + 2 * i > last_key) e0 = 0.f;
+                    if (key0 + 2 * i + 1 > last_key) e1 = 0.f;
                 }
-                // piece c4 of P lands on columns [16 c4, 16 c4 + 16), all of them already read above
-                tc::tmem_st16(tS + c4 * 16, pk);
+                if (i & 1) rowsum2 += e0 + e1; else rowsum += e0 + e1;
+                v[i] = pack_half2(e0, e1);
+            }
+            rowsum += rowsum2;
+            {
+                const uint32_t(&p0)[32] = *reinterpret_cast<const uint32_t(*)[32]>(&v[0]);
+                const uint32_t(&p1)[32] = *reinterpret_cast<const uint32_t(*)[32]>(&v[32]);
+                tc::tmem_st32(tS, p0);
+                tc::tmem_st32(tS + 32, p1);
             }
             l_run += rowsum;
             tc::tmem_st_wait();
@@ -374,62 +402,58 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 ++raw_issued;
             }
         }
-    } else {
-        // =========================================================== MMA issue (one thread)
+    } else if (warp < 15) {
+        // =========================================================== MMA issue for query tile t (one thread each);
+        //                                                             warp 15 only fills its warp group
+        const int t = warp - 13;
         if (lane == 0 && T > 0) {
             constexpr uint32_t idesc_qk = tc::instr_desc(1, 0, 0, false, false, 128, 128);   // f32 <- f16 x f16, both K-major
             constexpr uint32_t idesc_pv = tc::instr_desc(1, 0, 0, false, true, 128, 128);    // B (V) is MN-major
-            auto issue_qk = [&](int t) {   // S_t = Q_t . K^T
+            const int Tmine = t ? T1 : T0;
+            // Operand descriptors are built once; an MMA step only adds a constant to the address field.
+            const uint64_t dq = tc::smem_desc(sbase + pfl::kQ + (uint32_t)t * 32768u, 16, 1024, tc::kSwizzle128B);
+            const uint64_t dk = tc::smem_desc(sbase + pfl::kKf, 16, 1024, tc::kSwizzle128B);
+            const uint64_t dv = tc::smem_desc(sbase + pfl::kVf, 16384, 1024, tc::kSwizzle128B);
+            const uint32_t dS = tmem + kPfTmemS + (uint32_t)t * 128u, dO = tmem + kPfTmemO + (uint32_t)t * 128u;
+            auto issue_qk = [&]() {   // S_t = Q_t . K^T
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t koff = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
-                    const uint64_t a = tc::smem_desc(sbase + pfl::kQ + (uint32_t)t * 32768u + koff, 16, 1024, tc::kSwizzle128B);
-                    const uint64_t bk = tc::smem_desc(sbase + pfl::kKf + koff, 16, 1024, tc::kSwizzle128B);
-                    tc::mma_f16(tmem + kPfTmemS + (uint32_t)t * 128u, a, bk, idesc_qk, ks > 0);
+                    // dims [16 ks, 16 ks + 16): half ks / 4 of the tile (16 KB apart), 32 bytes per step inside the swizzle span
+                    const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+                    tc::mma_f16(dS, dq + koff, dk + koff, idesc_qk, ks > 0);
                 }
                 tc::commit(bar(pfl::S_FULL, t));
             };
-            auto issue_pv = [&](int t, bool first) {   // O_t (+)= P_t . V
+            auto issue_pv = [&](bool first) {   // O_t (+)= P_t . V
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t bv = tc::smem_desc(sbase + pfl::kVf + ks * 2048, 16384, 1024, tc::kSwizzle128B);
-                    tc::mma_f16_ts(tmem + kPfTmemO + (uint32_t)t * 128u, tmem + kPfTmemS + (uint32_t)t * 128u + ks * 8, bv,
-                                   idesc_pv, !first || ks > 0);
-                }
+                for (int ks = 0; ks < 8; ++ks)   // keys [16 ks, 16 ks + 16): 2 KB further down the V tile, 8 columns of P
+                    tc::mma_f16_ts(dO, dS + ks * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, !first || ks > 0);
                 tc::commit(bar(pfl::O_DONE, t));
             };
-            if (T0 > 0) wait(bar(pfl::Q_FULL, 0), 0);
-            if (T1 > 0) wait(bar(pfl::Q_FULL, 1), 0);
+            // Both threads walk all T key tiles and hand every K / V buffer back (two arrivals free it), also
+            // for the tiles their query tile does not see: a thread never runs ahead of the fill it waits for.
+            if (Tmine > 0) wait(bar(pfl::Q_FULL, t), 0);
             wait(bar(pfl::KF_FULL, 0), 0);
             tc::fence_after_sync();
-            if (T0 > 0) issue_qk(0);
-            if (T1 > 0) issue_qk(1);
+            if (Tmine > 0) issue_qk();
             tc::commit(bar(pfl::KF_EMPTY, 0));
             for (int j = 0; j < T; ++j) {
-                const uint32_t ph = (uint32_t)j & 1u, phn = ph ^ 1u;
-                const bool a0 = j < T0, a1 = j < T1, n0 = j + 1 < T0, n1 = j + 1 < T1;
+                const uint32_t ph = (uint32_t)j & 1u;
                 wait(bar(pfl::VF_FULL, 0), ph);
-                if (a0) {
-                    wait(bar(pfl::P_FULL, 0), ph);
+                if (j < Tmine) {
+                    wait(bar(pfl::P_FULL, t), ph);
                     tc::fence_after_sync();
-                    issue_pv(0, j == 0);
-                }
-                if (n0 || n1) wait(bar(pfl::KF_FULL, 0), phn);
-                if (n0) {
-                    tc::fence_after_sync();
-                    issue_qk(0);
-                }
-                if (a1) {
-                    wait(bar(pfl::P_FULL, 1), ph);
-                    tc::fence_after_sync();
-                    issue_pv(1, j == 0);
+                    issue_pv(j == 0);
                 }
                 tc::commit(bar(pfl::VF_EMPTY, 0));
-                if (n1) {
-                    tc::fence_after_sync();
-                    issue_qk(1);
+                if (j + 1 < T) {
+                    wait(bar(pfl::KF_FULL, 0), ph ^ 1u);
+                    if (j + 1 < Tmine) {
+                        tc::fence_after_sync();
+                        issue_qk();
+                    }
+                    tc::commit(bar(pfl::KF_EMPTY, 0));
                 }
-                if (n0 || n1) tc::commit(bar(pfl::KF_EMPTY, 0));
             }
         }
     }

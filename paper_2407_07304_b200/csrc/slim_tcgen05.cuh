@@ -113,6 +113,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+// This warp's 32 lanes x 8 consecutive 32-bit columns, store.
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
 // This warp's 32 lanes x 16 consecutive 32-bit columns, store.
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
 {
@@ -139,17 +146,23 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t mbar_smem, uint32
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(mbar_smem), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity; false if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar_smem, uint32_t parity, uint32_t max_tries = (1u << 18))
+// Bounded wait for the phase with the given parity; false if the limit ran out (or, when `abort` is
+// given, if another thread of the block has raised it).  Each try lets the hardware suspend the thread
+// for up to kWaitHintNs, so a waiting warp does not compete for issue slots; the bound is
+// max_tries * kWaitHintNs at most (about 0.13 s with the defaults).
+constexpr uint32_t kWaitHintNs = 512;
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar_smem, uint32_t parity, uint32_t max_tries = (1u << 18),
+                                          const volatile int *abort = nullptr)
 {
     for (uint32_t i = 0; i < max_tries; ++i) {
         uint32_t done;
         asm volatile(
-            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}\n"
+            "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}\n"
             : "=r"(done)
-            : "r"(mbar_smem), "r"(parity)
+            : "r"(mbar_smem), "r"(parity), "r"(kWaitHintNs)
             : "memory");
         if (done) return true;
+        if (abort != nullptr && (i & 15u) == 15u && *abort != 0) return false;
     }
     return false;
 }
