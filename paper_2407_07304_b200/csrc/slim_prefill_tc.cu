@@ -12,10 +12,9 @@
 //   warps 8-11  dequantise in registers (the hybrid-dtype step of Section 2.2): INT8 codes -> fp16
 //               code * scale / 2^e, written in the swizzled layout the tensor cores read (one K and
 //               one V operand buffer; a buffer is refilled as soon as the MMAs that read it are done)
-//   warps 13,14 one MMA-issuing thread per query tile, each in the order  P_t.V(j), Q_t.K(j+1)^T:
+//   warp 13     one thread issues tcgen05.mma in the order  P0.V(j), Q0.K(j+1)^T, P1.V(j), Q1.K(j+1)^T:
 //               S_t = Q_t . K^T (both operands in shared memory), O_t += P_t . V (P read from tensor
-//               memory), fp32 accumulators in tensor memory.  Two threads so that neither tile waits for
-//               the other one's softmax.
+//               memory), fp32 accumulators in tensor memory
 //   warps 0-3   softmax of Q0, warps 4-7 softmax of Q1; thread = query row.  The whole 128-column score row is
 //               read into registers with one tcgen05.ld round trip (the softmax warps take registers from the
 //               other warp groups: setmaxnreg), then row maximum, exp2 -> fp16 P back to tensor memory and the
@@ -33,7 +32,7 @@
 
 namespace slim {
 
-constexpr int kPfThreads = 512;   // four warp groups: softmax 0, softmax 1, dequantisers, {loader, two MMA threads, one idle warp}
+constexpr int kPfThreads = 512;   // four warp groups: softmax 0, softmax 1, dequantisers, {loader, MMA thread, two idle warps}
 constexpr int kPfBM = 128, kPfBN = 128;
 constexpr int kPfRows = 2 * kPfBM;             // query rows per block
 constexpr int kPfRawStages = 5;
@@ -132,9 +131,9 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             tc::mbar_init(bar(pfl::RAW_EMPTY, i), 128);
         }
         tc::mbar_init(bar(pfl::KF_FULL, 0), 128);
-        tc::mbar_init(bar(pfl::KF_EMPTY, 0), 2);   // both MMA threads are done with the K tile
+        tc::mbar_init(bar(pfl::KF_EMPTY, 0), 1);
         tc::mbar_init(bar(pfl::VF_FULL, 0), 128);
-        tc::mbar_init(bar(pfl::VF_EMPTY, 0), 2);
+        tc::mbar_init(bar(pfl::VF_EMPTY, 0), 1);
         for (int t = 0; t < 2; ++t) {
             tc::mbar_init(bar(pfl::S_FULL, t), 1);
             tc::mbar_init(bar(pfl::P_FULL, t), 128);
@@ -237,20 +236,19 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 tc::tmem_ld32(tS + 96, v3);
                 tc::tmem_ld_wait();
             }
-            float mx = -INFINITY;
-            if (diag) {
+            // causal mask: only warps that touch the diagonal execute it (minus infinity becomes weight 0 below)
+            if (__any_sync(0xffffffffu, diag)) {
 #pragma unroll
                 for (int i = 0; i < 128; ++i)
-                    if (key0 + i <= last_key) mx = fmaxf(mx, __uint_as_float(v[i]));
-            } else {
-                float mx2 = -INFINITY;   // two chains
-#pragma unroll
-                for (int i = 0; i < 128; i += 4) {
-                    mx = pf_max3(mx, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-                    mx2 = pf_max3(mx2, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-                }
-                mx = fmaxf(mx, mx2);
+                    if (key0 + i > last_key) v[i] = 0xFF800000u;
             }
+            float mx = -INFINITY, mx2 = -INFINITY;   // two chains
+#pragma unroll
+            for (int i = 0; i < 128; i += 4) {
+                mx = pf_max3(mx, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                mx2 = pf_max3(mx2, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            }
+            mx = fmaxf(mx, mx2);
             const float mt = (mx == -INFINITY) ? -INFINITY : mx * c;
             // the reference maximum only moves when the tile's exceeds it by more than the threshold
             const bool grow = (j == 0) ? true : (mt > m_run + kPfRescaleThreshold);
@@ -277,12 +275,8 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             float rowsum = 0.f, rowsum2 = 0.f;
 #pragma unroll
             for (int i = 0; i < 64; ++i) {
-                float e0 = pf_exp2(fmaf(__uint_as_float(v[2 * i]), c, bias));
-                float e1 = pf_exp2(fmaf(__uint_as_float(v[2 * i + 1]), c, bias));
-                if (diag) {
-                    if (key0 + 2 * i > last_key) e0 = 0.f;
-                    if (key0 + 2 * i + 1 > last_key) e1 = 0.f;
-                }
+                const float e0 = pf_exp2(fmaf(__uint_as_float(v[2 * i]), c, bias));
+                const float e1 = pf_exp2(fmaf(__uint_as_float(v[2 * i + 1]), c, bias));
                 if (i & 1) rowsum2 += e0 + e1; else rowsum += e0 + e1;
                 v[i] = pack_half2(e0, e1);
             }
@@ -402,58 +396,68 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 ++raw_issued;
             }
         }
-    } else if (warp < 15) {
-        // =========================================================== MMA issue for query tile t (one thread each);
-        //                                                             warp 15 only fills its warp group
-        const int t = warp - 13;
+    } else if (warp == 13) {
+        // =========================================================== MMA issue (one thread); warps 14, 15 only fill the warp group
         if (lane == 0 && T > 0) {
             constexpr uint32_t idesc_qk = tc::instr_desc(1, 0, 0, false, false, 128, 128);   // f32 <- f16 x f16, both K-major
             constexpr uint32_t idesc_pv = tc::instr_desc(1, 0, 0, false, true, 128, 128);    // B (V) is MN-major
-            const int Tmine = t ? T1 : T0;
             // Operand descriptors are built once; an MMA step only adds a constant to the address field.
-            const uint64_t dq = tc::smem_desc(sbase + pfl::kQ + (uint32_t)t * 32768u, 16, 1024, tc::kSwizzle128B);
+            const uint64_t dq0 = tc::smem_desc(sbase + pfl::kQ, 16, 1024, tc::kSwizzle128B);
+            const uint64_t dq1 = tc::smem_desc(sbase + pfl::kQ + 32768u, 16, 1024, tc::kSwizzle128B);
             const uint64_t dk = tc::smem_desc(sbase + pfl::kKf, 16, 1024, tc::kSwizzle128B);
             const uint64_t dv = tc::smem_desc(sbase + pfl::kVf, 16384, 1024, tc::kSwizzle128B);
-            const uint32_t dS = tmem + kPfTmemS + (uint32_t)t * 128u, dO = tmem + kPfTmemO + (uint32_t)t * 128u;
-            auto issue_qk = [&]() {   // S_t = Q_t . K^T
+            auto issue_qk = [&](int t) {   // S_t = Q_t . K^T
+                const uint64_t dq = t ? dq1 : dq0;
+                const uint32_t d = tmem + kPfTmemS + (uint32_t)t * 128u;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     // dims [16 ks, 16 ks + 16): half ks / 4 of the tile (16 KB apart), 32 bytes per step inside the swizzle span
                     const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-                    tc::mma_f16(dS, dq + koff, dk + koff, idesc_qk, ks > 0);
+                    tc::mma_f16(d, dq + koff, dk + koff, idesc_qk, ks > 0);
                 }
                 tc::commit(bar(pfl::S_FULL, t));
             };
-            auto issue_pv = [&](bool first) {   // O_t (+)= P_t . V
+            auto issue_pv = [&](int t, bool first) {   // O_t (+)= P_t . V
+                const uint32_t d = tmem + kPfTmemO + (uint32_t)t * 128u, a = tmem + kPfTmemS + (uint32_t)t * 128u;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)   // keys [16 ks, 16 ks + 16): 2 KB further down the V tile, 8 columns of P
-                    tc::mma_f16_ts(dO, dS + ks * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, !first || ks > 0);
+                    tc::mma_f16_ts(d, a + ks * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, !first || ks > 0);
                 tc::commit(bar(pfl::O_DONE, t));
             };
-            // Both threads walk all T key tiles and hand every K / V buffer back (two arrivals free it), also
-            // for the tiles their query tile does not see: a thread never runs ahead of the fill it waits for.
-            if (Tmine > 0) wait(bar(pfl::Q_FULL, t), 0);
+            if (T0 > 0) wait(bar(pfl::Q_FULL, 0), 0);
+            if (T1 > 0) wait(bar(pfl::Q_FULL, 1), 0);
             wait(bar(pfl::KF_FULL, 0), 0);
             tc::fence_after_sync();
-            if (Tmine > 0) issue_qk();
+            if (T0 > 0) issue_qk(0);
+            if (T1 > 0) issue_qk(1);
             tc::commit(bar(pfl::KF_EMPTY, 0));
+            // The fixed order P0.V(j), Q0.K(j+1)^T, P1.V(j), Q1.K(j+1)^T keeps the two query tiles half a step
+            // apart, so that their softmax phases (which share the special-function units) alternate.
             for (int j = 0; j < T; ++j) {
-                const uint32_t ph = (uint32_t)j & 1u;
+                const uint32_t ph = (uint32_t)j & 1u, phn = ph ^ 1u;
+                const bool a0 = j < T0, a1 = j < T1, n0 = j + 1 < T0, n1 = j + 1 < T1;
                 wait(bar(pfl::VF_FULL, 0), ph);
-                if (j < Tmine) {
-                    wait(bar(pfl::P_FULL, t), ph);
+                if (a0) {
+                    wait(bar(pfl::P_FULL, 0), ph);
                     tc::fence_after_sync();
-                    issue_pv(j == 0);
+                    issue_pv(0, j == 0);
+                }
+                if (n0 || n1) wait(bar(pfl::KF_FULL, 0), phn);
+                if (n0) {
+                    tc::fence_after_sync();
+                    issue_qk(0);
+                }
+                if (a1) {
+                    wait(bar(pfl::P_FULL, 1), ph);
+                    tc::fence_after_sync();
+                    issue_pv(1, j == 0);
                 }
                 tc::commit(bar(pfl::VF_EMPTY, 0));
-                if (j + 1 < T) {
-                    wait(bar(pfl::KF_FULL, 0), ph ^ 1u);
-                    if (j + 1 < Tmine) {
-                        tc::fence_after_sync();
-                        issue_qk();
-                    }
-                    tc::commit(bar(pfl::KF_EMPTY, 0));
+                if (n1) {
+                    tc::fence_after_sync();
+                    issue_qk(1);
                 }
+                if (n0 || n1) tc::commit(bar(pfl::KF_EMPTY, 0));
             }
         }
     }
