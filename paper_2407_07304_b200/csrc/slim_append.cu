@@ -9,9 +9,10 @@
 //  * code = round_half_even(127 x / amax) on the exact ratio.  The fast path multiplies by the
 //    correctly rounded 127 / amax and rounds with the 1.5 * 2^23 trick; the product is within 2^-16 of
 //    the exact ratio, so whenever it lies further than 2^-10 from a rounding tie the result is the
-//    exact one.  Elements nearer to a tie (0.5 % of them, most of them exact ties of the coarse bf16
-//    grid) are redone with the IEEE division of the exact product 127 x by amax, which decides the
-//    tie correctly.  Codes and scales are therefore reproducible bit for bit.
+//    exact one.  For the elements nearer to a tie (0.3 % of them, most of them exact ties of the coarse
+//    bf16 grid) the exact residual 127 x - c * amax is compared with amax / 2, which decides the tie
+//    correctly; a warp takes that path only when one of its lanes needs it.  Codes and scales are
+//    therefore reproducible bit for bit.
 #include "slim_common.cuh"
 
 namespace slim {
@@ -34,8 +35,10 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
     const int kv = blockIdx.z;
     const int hw = threadIdx.x >> 4, l = threadIdx.x & 15;
     const int row0 = __ldg(cu_new + b);
-    const long long n_rows = (long long)(__ldg(cu_new + b + 1) - row0) * Hkv;
-    const long long first = (long long)blockIdx.x * kAppendRowsPerBlock;
+    // 32-bit row arithmetic (the host checks that max_new * Hkv fits): 64-bit divisions would cost more
+    // instructions than the quantiser itself
+    const int n_rows = (__ldg(cu_new + b + 1) - row0) * Hkv;
+    const int first = (int)blockIdx.x * kAppendRowsPerBlock;
     if (first >= n_rows) return;
     const int start = __ldg(start_pos + b);
     const uint4 *src = reinterpret_cast<const uint4 *>((kv ? v_new : k_new) + (size_t)row0 * Hkv * kHeadDim);
@@ -45,13 +48,13 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
     int page[kAppendRowsPerGroup], head[kAppendRowsPerGroup], slot[kAppendRowsPerGroup];
 #pragma unroll
     for (int i = 0; i < kAppendRowsPerGroup; ++i) {
-        const long long r = first + i * 16 + hw;     // the block's half-warps cover 16 consecutive rows per step
+        const int r = first + i * 16 + hw;     // the block's half-warps cover 16 consecutive rows per step
         page[i] = -1;
         raw[i] = make_uint4(0, 0, 0, 0);
         if (r < n_rows) {
-            raw[i] = __ldg(src + r * 16 + l);
-            const int tok = (int)(r / Hkv);
-            head[i] = (int)(r - (long long)tok * Hkv);
+            raw[i] = __ldg(src + (size_t)r * 16 + l);
+            const int tok = (int)((unsigned)r / (unsigned)Hkv);
+            head[i] = r - tok * Hkv;
             const int pos = start + tok;
             slot[i] = pos & (kPageTokens - 1);
             const int page_idx = pos >> 7;
@@ -74,25 +77,26 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));   // within the 16 lanes
 
-        uint32_t tb[8];   // low byte = the code in two's complement
-        if (amax > 0.f) {
-            const float inv = __fdiv_rn(127.f, amax);
+        uint32_t tb[8];   // 0x4B400000 + code: the low byte is the code in two's complement
+        const float inv = (amax > 0.f) ? __fdiv_rn(127.f, amax) : 0.f;   // an all-zero row gets codes 0
+        const float half = 0.5f * amax;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const float q = x[k] * inv;
-                float t = q + kRoundMagic;
-                const float d = fabsf(q - (t - kRoundMagic));
-                if (d > 0.5f - 0x1p-10f) {
-                    // near a rounding tie: 127 * x is exact in fp32 for a bf16 x, the quotient is correctly rounded
-                    int c = __float2int_rn(__fdiv_rn(127.f * x[k], amax));
-                    c = max(-127, min(127, c));
-                    t = __int_as_float(0x4B400000 + c);
-                }
-                tb[k] = __float_as_uint(t);
+        for (int k = 0; k < 8; ++k) {
+            const float q = x[k] * inv;
+            const float t = q + kRoundMagic;
+            const float c0 = t - kRoundMagic;                    // q rounded to the nearest integer, ties to even
+            tb[k] = __float_as_uint(t);
+            const bool near = fabsf(q - c0) > 0.5f - 0x1p-10f;   // 0.3 % of the elements
+            if (__any_sync(0xffffffffu, near)) {
+                // Near a rounding tie the approximate quotient may have picked the wrong neighbour.  The residual
+                // 127 x - c0 * amax is exact in fp32 (127 x has 15 significant bits, c0 * amax at most 15, and they
+                // are within a factor 2^9 of each other when c0 != 0), so comparing it with amax / 2 decides exactly.
+                const float e = fmaf(-c0, amax, 127.f * x[k]);
+                const bool odd = (tb[k] & 1u) != 0u;
+                const int up = (e > half || (e == half && odd)) ? 1 : 0;
+                const int dn = (e < -half || (e == -half && odd)) ? 1 : 0;
+                if (near) tb[k] += (uint32_t)(up - dn);
             }
-        } else {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) tb[k] = 0u;
         }
         if (page[i] >= 0 && page[i] < num_pages) {
             uint2 pk;
@@ -111,7 +115,7 @@ int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, c
 {
     const long long rows = (long long)max_new * c->num_kv_heads;
     const long long blocks = (rows + kAppendRowsPerBlock - 1) / kAppendRowsPerBlock;
-    if (blocks > 0x7FFFFFFFLL) return SLIM_ERR_UNSUPPORTED;
+    if (rows > 0x7FFFFF00LL) return SLIM_ERR_UNSUPPORTED;   // the kernel indexes rows with 32-bit integers
     dim3 grid((unsigned)blocks, (unsigned)B, 2);
     slim_append_kernel<<<grid, kAppendThreads, 0, stream>>>(
         c->codes, c->scales, c->block_table, static_cast<const __nv_bfloat16 *>(k_new),
