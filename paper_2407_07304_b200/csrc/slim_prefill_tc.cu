@@ -74,6 +74,29 @@ __device__ __forceinline__ float pf_exp2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
 }
+// packed fp32 pairs in a 64-bit register (two values per instruction)
+__device__ __forceinline__ uint64_t pf_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void pf_unpack(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t pf_fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t pf_add2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 __device__ __forceinline__ float pf_max3(float a, float b, float c)
 {
     float m;
@@ -272,15 +295,20 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             if (grow) m_run = mt;
             const float bias = (m_run == -INFINITY) ? 0.f : -m_run;
             // ---- P = 2^(s - m) as fp16 pairs, packed in place, into the first 64 columns of the score buffer
-            float rowsum = 0.f, rowsum2 = 0.f;
+            // (packed fp32 arithmetic: one fused multiply-add and one add per pair of scores)
+            const uint64_t c2 = pf_pack(c, c), bias2 = pf_pack(bias, bias);
+            uint64_t sum2a = 0ull, sum2b = 0ull;
 #pragma unroll
             for (int i = 0; i < 64; ++i) {
-                const float e0 = pf_exp2(fmaf(__uint_as_float(v[2 * i]), c, bias));
-                const float e1 = pf_exp2(fmaf(__uint_as_float(v[2 * i + 1]), c, bias));
-                if (i & 1) rowsum2 += e0 + e1; else rowsum += e0 + e1;
+                float x0, x1;
+                pf_unpack(pf_fma2(pf_pack(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), c2, bias2), x0, x1);
+                const float e0 = pf_exp2(x0), e1 = pf_exp2(x1);
+                if (i & 1) sum2b = pf_add2(sum2b, pf_pack(e0, e1)); else sum2a = pf_add2(sum2a, pf_pack(e0, e1));
                 v[i] = pack_half2(e0, e1);
             }
-            rowsum += rowsum2;
+            float rowsum, rowsum_hi;
+            pf_unpack(pf_add2(sum2a, sum2b), rowsum, rowsum_hi);
+            rowsum += rowsum_hi;
             {
                 const uint32_t(&p0)[32] = *reinterpret_cast<const uint32_t(*)[32]>(&v[0]);
                 const uint32_t(&p1)[32] = *reinterpret_cast<const uint32_t(*)[32]>(&v[32]);
