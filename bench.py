@@ -40,6 +40,22 @@ def _peaks():
     return 6650.0, 1590.0, "fallback"
 
 
+def max_over_ranks(ms, world, device):
+    """The slowest rank's time (every rank gets it); plain value when there is one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank_per_step, steps, world, ms_max):
+    """Aggregate units/s of `world` ranks that each did the same work, timed by the slowest rank."""
+    return world * units_per_rank_per_step * steps / (ms_max * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi clock/throttle sampling while the timed region runs (read-only queries)."""
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -223,11 +239,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
         barrier()
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ms, world, dev)
 
     for i in range(max(3, args.warmup)):
         step(i)
@@ -285,7 +297,7 @@ def run_ours(args, rank, world, local_rank):
     h2d = (B * Hq + 2 * B * Hkv) * 128 * 2
     d2h = B * Hq * 128 * 2
     line = {
-        "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_rate(B, args.steps, world, ms_total), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8 (tcgen05 kind::i8 MMA, s32 accumulate; fp32 softmax)",
         "data": "synthetic",
@@ -299,7 +311,7 @@ def run_ours(args, rank, world, local_rank):
                      "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_8tbs": achieved / 8000.0, "bytes_per_launch": split_bytes,
                      "avg_launch_ms": split_avg_ms, "min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
-        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": whole_job_rate(B, args.steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same)},
         "gpu_launches": 3 * args.steps,
         "clocks": clocks,
@@ -313,9 +325,9 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
-# dram bytes read + written by one slim_decode_split_kernel launch on this workload, from the ncu
-# capture summarised under profiles/ ; None until a capture of the current kernel exists.
-TRAFFIC_PER_LAUNCH = 284.74e6
+# dram bytes read + written by one slim_decode_stream_kernel launch on this workload (279.68 MB read,
+# 6.07 MB written), from the ncu capture summarised under profiles/.
+TRAFFIC_PER_LAUNCH = 285.75e6
 
 
 def extra_numbers(slim, workloads, dev):
@@ -356,14 +368,67 @@ def extra_numbers(slim, workloads, dev):
     flops = 4 * 128 * w3.Hq * S * (S + 1) // 2
     append_bytes = S * w3.Hkv * (2 * 256 + ROW_BYTES)
     hbm_peak, _, _ = _peaks()
-    return {
+    del run, q, out, k_new, v_new
+
+    def decode_numbers(index, copies, label):
+        """slim_attn_decode (split + merge) of workload `index` at its final context, cache pre-filled untimed."""
+        w = workloads.make_workload(index)
+        runs = []
+        for _ in range(copies):
+            r = LayerRun(w, device=dev)
+            ctx = [w.total_len(b) - w.decode_steps for b in range(w.B)]
+            r.append(ctx)
+            r.append([1] * w.B)
+            runs.append(r)
+        qd = w.q_decode[0].to(dev).contiguous()
+        od = torch.empty_like(qd)
+        kvl = torch.tensor(runs[0].pos, dtype=torch.int32, device=dev)
+        mk = max(runs[0].pos)
+        it = [0]
+
+        def dec():
+            c = runs[it[0] % copies]
+            it[0] += 1
+            slim.slim_attn_decode(c.cache, qd, od, kvl, w.B, mk, w.Hq, w.sm_scale, runs[0].ws_decode, stream)
+
+        ms = time_it(dec, 50)
+        nbytes = sum(runs[0].pos) * w.Hkv * ROW_BYTES + 2 * w.B * w.Hq * 256
+        return {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
+                "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "cache": label}
+
+    def prefill_numbers(index):
+        w = workloads.make_workload(index)
+        r = LayerRun(w, device=dev)
+        n = w.prefill_len[0]
+        r.append(w.prefill_len)
+        cu5 = torch.tensor([0, n], dtype=torch.int32, device=dev)
+        kv5 = torch.tensor([n], dtype=torch.int32, device=dev)
+        q5 = w.q_prefill[0].to(dev).contiguous()
+        o5 = torch.empty_like(q5)
+
+        def pf():
+            slim.slim_attn_prefill(r.cache, q5, o5, cu5, kv5, 1, n, n, w.Hq, w.sm_scale, r.ws_prefill, stream)
+
+        ms = time_it(pf, 3)
+        fl = 4 * 128 * w.Hq * n * (n + 1) // 2
+        return {"workload": w.name, "ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
+                "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
+
+    more = {}
+    if not os.environ.get("SLIM_BENCH_SHORT"):
+        more = {"decode_c4": decode_numbers(4, 2, "two cache copies rotated (2 x 173 MB > L2)"),
+                "decode_c5": decode_numbers(5, 1, "17 MB, L2-resident: a latency number, not an HBM number"),
+                "decode_c1": decode_numbers(1, 1, "2 MB, L2-resident: a latency number, not an HBM number"),
+                "prefill_c5": prefill_numbers(5),
+                "prefill_c1": prefill_numbers(1)}
+    return {**more, **{
         "prefill_c3": {"workload": w3.name, "ms": ms_prefill, "tflops": flops / (ms_prefill * 1e-3) / 1e12,
                        "frac_of_bf16_peak": flops / (ms_prefill * 1e-3) / 1e12 / bf16_peak,
                        "peak_tflops": bf16_peak, "peak_kind": f"of {peak_kind}",
                        "tokens_per_s_with_append": S / ((ms_prefill + ms_append) * 1e-3)},
         "append_c3": {"ms": ms_append, "gbs": append_bytes / (ms_append * 1e-3) / 1e9,
                       "frac_of_hbm_peak": append_bytes / (ms_append * 1e-3) / 1e9 / hbm_peak},
-    }
+    }}
 
 
 def main():

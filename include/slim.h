@@ -118,7 +118,8 @@ int slim_kv_append(const slim_cache_t *cache, const void *k_new, const void *v_n
  *   max_q, max_kv  upper bounds on q_len and kv_len (size the launch)
  *   workspace      device scratch of at least
  *                  slim_workspace_bytes(SLIM_PHASE_PREFILL, ...) bytes (may be
- *                  NULL when that size is 0)
+ *                  NULL when that size is 0); its first 16 bytes are the status
+ *                  word (see slim_read_status) and should be zero
  */
 int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out,
                       const int32_t *cu_q, const int32_t *kv_len,
@@ -137,7 +138,8 @@ int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out,
  *   kv_len   device int32 [B];  max_kv upper bound on kv_len (sizes the launch)
  *   workspace device scratch of at least
  *             slim_workspace_bytes(SLIM_PHASE_DECODE, ...) bytes, 16-byte
- *             aligned; contents need not be initialised
+ *             aligned; only its first 16 bytes (the status word, see
+ *             slim_read_status) need to be zero, the rest need not be initialised
  */
 int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out,
                      const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
@@ -218,6 +220,16 @@ size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
 int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
                             const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
                             void *stream);
+
+/*
+ * Device-side waits are bounded.  The attention kernels wait on hardware barriers (TMA copies, tensor-core
+ * completion); every such wait gives up after a fixed number of tries, and a kernel whose wait ran out
+ * stores SLIM_ERR_TIMEOUT in the first word of its workspace and finishes with undefined output instead of
+ * hanging.  slim_read_status synchronises `stream`, reads that word (host <- device) and returns SLIM_OK
+ * or SLIM_ERR_TIMEOUT.  The kernels never clear the word: zero the first 16 bytes of a workspace once
+ * after allocating it.
+ */
+int slim_read_status(const void *workspace, void *stream);
 
 /* Scratch bytes needed by a phase (SLIM_PHASE_*) for the given shape; 0 on invalid arguments. */
 size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q, int32_t max_kv);

@@ -25,7 +25,7 @@ PAGE_TOKENS = 128
 
 EXPORTS = (
     "slim_kv_append", "slim_attn_prefill", "slim_attn_decode", "slim_attn_decode_split",
-    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step_host", "slim_step_staging_bytes", "slim_workspace_bytes",
+    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -84,6 +84,8 @@ def lib():
         L.slim_decode_step_host.restype = ctypes.c_int
         L.slim_step_staging_bytes.argtypes = [I, I, I]
         L.slim_step_staging_bytes.restype = Z
+        L.slim_read_status.argtypes = [P, P]
+        L.slim_read_status.restype = ctypes.c_int
         L.slim_workspace_bytes.argtypes = [I, I, I, I, I, I]
         L.slim_workspace_bytes.restype = Z
         L.slim_cache_code_bytes.argtypes = [I, I]
@@ -200,6 +202,11 @@ def slim_decode_step_host(cache, q_host, k_new_host, v_new_host, out_host, stagi
                                      _ptr(kv_len), B, max_kv, Hq, sm_scale, _ptr(workspace), _nbytes(workspace),
                                      _stream(stream))
     _check(rc, "slim_decode_step_host")
+
+
+def slim_read_status(workspace, stream=None):
+    """Synchronises the stream and returns SLIM_OK or SLIM_ERR_TIMEOUT (a bounded device-side wait ran out)."""
+    return lib().slim_read_status(_ptr(workspace), _stream(stream))
 
 
 def slim_step_staging_bytes(B, Hq, Hkv):

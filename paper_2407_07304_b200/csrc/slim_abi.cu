@@ -1,6 +1,4 @@
 // C ABI of the library (declared in include/slim.h): argument validation and dispatch.
-#include <stdlib.h>
-
 #include "slim_common.cuh"
 
 #define SLIM_EXPORT extern "C" __attribute__((visibility("default")))
@@ -25,8 +23,6 @@ size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                       int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 size_t prefill_workspace_bytes();
-int launch_prefill_mma(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
-                       int B, int max_q, int Hq, float sm_scale, cudaStream_t stream);
 
 static int check_cache(const slim_cache_t *c)
 {
@@ -71,12 +67,6 @@ SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void
     if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
     const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
-    // SLIM_PREFILL_IMPL=mma selects the warp-level MMA kernel (kept for cross-checks); default is tcgen05
-    static const bool use_mma = [] {
-        const char *e = getenv("SLIM_PREFILL_IMPL");
-        return e != nullptr && e[0] == 'm';
-    }();
-    if (use_mma) return launch_prefill_mma(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, (cudaStream_t)stream);
     return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream);
 }
 
@@ -179,6 +169,15 @@ SLIM_EXPORT size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, in
     if (phase == SLIM_PHASE_DECODE) return decode_workspace_bytes(B, Hq, Hkv, max_kv);
     if (phase == SLIM_PHASE_PREFILL) return prefill_workspace_bytes();
     return 0;
+}
+
+SLIM_EXPORT int slim_read_status(const void *workspace, void *stream)
+{
+    if (workspace == nullptr) return SLIM_ERR_INVALID_ARG;
+    int word = 0;
+    SLIM_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    SLIM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return (word == 0) ? SLIM_OK : SLIM_ERR_TIMEOUT;
 }
 
 SLIM_EXPORT size_t slim_cache_code_bytes(int32_t num_pages, int32_t num_kv_heads)

@@ -20,7 +20,6 @@ struct DecodeParams {
 
 constexpr size_t kDecodeStatusBytes = 16;   // status word + padding in front of the partials
 
-int launch_decode_split_tc(const DecodeParams &p, int B, cudaStream_t stream);
 int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int B, cudaStream_t stream);
 
 }  // namespace slim

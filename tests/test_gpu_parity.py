@@ -209,3 +209,49 @@ def test_bad_arguments_are_rejected_on_the_host():
         slim.slim_attn_decode(run.cache, q, q.clone(), kvl, 1, 100000, 4, 1.0, run.ws_decode)  # beyond the page table
     assert e.value.code == slim.SLIM_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+# ---------------------------------------------------------------- more decode shapes and the host-step entry point
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (16, 1)])
+def test_decode_tail_lengths(Hq, Hkv):
+    # lengths around every boundary of the streaming kernel: the 16-row boxes of a ragged tile, the
+    # 128-token tile, the 256-token chunk; one and sixteen query heads per kv head (both consumer layouts)
+    lens = [1, 15, 16, 17, 31, 127, 128, 129, 144, 255, 256, 257, 272, 383, 511, 513]
+    B = len(lens)
+    _check(_custom(B, Hq, Hkv, [0] * B, [n - 1 for n in lens], 1, 700 + Hq))
+
+
+def test_status_words_stay_clear():
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = workloads.make_workload(1, shrink=2)
+    run, _, _ = harness.run_workload(w, decode_steps={0})
+    assert slim.slim_read_status(run.ws_decode) == slim.SLIM_OK
+    assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
+
+
+def test_decode_step_from_host_buffers():
+    # slim_decode_step_host: H2D copies, append, split + merge, D2H copy on one stream
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = workloads.make_workload(4, shrink=16)
+    run = harness.LayerRun(w)
+    run.append(w.bulk_len)
+    dev = run.device
+    B, Hq, Hkv = w.B, w.Hq, w.Hkv
+    ctx = list(run.pos)
+    k_new = torch.stack([w.k[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
+    v_new = torch.stack([w.v[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
+    q = w.q_decode[0].contiguous().pin_memory()
+    out = torch.empty_like(q).pin_memory()
+    staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
+    cu_new = torch.arange(B + 1, dtype=torch.int32, device=dev)
+    start = torch.tensor(ctx, dtype=torch.int32, device=dev)
+    kv_len = start + 1
+    slim.slim_decode_step_host(run.cache, q, k_new, v_new, out, staging, cu_new, start, kv_len, B, max(ctx) + 1, Hq,
+                               w.sm_scale, run.ws_decode)
+    torch.cuda.synchronize()
+    run.pos = [c + 1 for c in ctx]
+    oc = _oracle_cache(w)
+    _assert_cache_bits(run, oc)
+    for b in range(B):
+        want = so.attention(bf16_bits(w.q_decode[0, b:b + 1]), *oc[b], ctx[b] + 1, w.sm_scale)
+        _assert_close(out[b:b + 1], want, f"host step seq {b}")
