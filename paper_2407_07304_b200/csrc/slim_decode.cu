@@ -14,43 +14,42 @@ constexpr int kChunkTok = 256;   // tokens per partial result (two pages)
 
 // Second pass: log-sum-exp merge of a row's chunk partials,
 //   M = max m_c;  l = sum l_c 2^(m_c - M);  o = sum O_c 2^(m_c - M) / l.
-// One block of 128 threads per (sequence, query head) row; thread = head dim.  The chunk weights go
-// through shared memory 128 at a time, so that the loads of the partial outputs (512 contiguous bytes
-// per chunk across the block) are independent of one another and many are in flight - a long sequence
-// has hundreds of chunks per row.
-constexpr int kMergeThreads = 128;
-
-__device__ __forceinline__ float merge_block_reduce(float v, bool is_max, float *red4, int tid)
-{
-    v = is_max ? warp_max(v) : warp_sum(v);
-    __syncthreads();                       // red4 may still be read from an earlier call
-    if ((tid & 31) == 0) red4[tid >> 5] = v;
-    __syncthreads();
-    return is_max ? fmaxf(fmaxf(red4[0], red4[1]), fmaxf(red4[2], red4[3])) : (red4[0] + red4[1]) + (red4[2] + red4[3]);
-}
-
-__global__ void __launch_bounds__(kMergeThreads)
+// One block per (sequence, query head) row: GROUPS groups of 128 threads (thread = head dim), group g takes
+// the chunks c = g mod GROUPS, so that a long sequence's hundreds of chunks are read with many independent
+// loads in flight (four groups); short rows use one group.  The chunk weights go through shared memory 128
+// at a time.
+template <int kMergeGroups>
+__global__ void __launch_bounds__(kMergeGroups * kHeadDim)
 slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                          const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
                          int B, int Hq, int n_chunks, int chunk_tokens)
 {
-    __shared__ float w_s[kMergeThreads];
-    __shared__ float red4[4];
+    constexpr int kMergeThreads = kMergeGroups * kHeadDim;
+    __shared__ float w_s[kHeadDim];
+    __shared__ float red[kMergeThreads / 32];
+    __shared__ float acc_s[kMergeGroups][kHeadDim];
     const int row = blockIdx.x;            // b * Hq + h
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, d = tid & (kHeadDim - 1), g = tid >> 7;
     pdl_wait();   // the split pass before this kernel must have finished writing the partials
     const int b = row / Hq;
     const int len = kv_len[b];
     const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
     const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_chunks;
     const float *po = part_o + (size_t)row * n_chunks * kHeadDim;
+    // ---- the row's maximum
     float M = -INFINITY;
     for (int c = tid; c < nc; c += kMergeThreads) M = fmaxf(M, ml[c].x);
-    M = merge_block_reduce(M, true, red4, tid);
+    M = warp_max(M);
+    if ((tid & 31) == 0) red[tid >> 5] = M;
+    __syncthreads();
+    M = red[0];
+#pragma unroll
+    for (int i = 1; i < kMergeThreads / 32; ++i) M = fmaxf(M, red[i]);
+    // ---- weighted sums, 128 chunks per round
     float acc = 0.f, lsum = 0.f;
-    for (int c0 = 0; c0 < nc; c0 += kMergeThreads) {
-        const int n = min(kMergeThreads, nc - c0);
-        __syncthreads();                   // the previous round's weights have been used
+    for (int c0 = 0; c0 < nc; c0 += kHeadDim) {
+        const int n = min(kHeadDim, nc - c0);
+        __syncthreads();                   // the previous round's weights (and the maxima) have been used
         if (tid < n) {
             const float2 v = ml[c0 + tid];
             const float w = exp2f(v.x - M);
@@ -58,21 +57,32 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
             lsum = fmaf(v.y, w, lsum);
         }
         __syncthreads();
-        const float *src = po + (size_t)c0 * kHeadDim + tid;
-        int c = 0;
-        for (; c + 4 <= n; c += 4) {
-            const float v0 = src[(size_t)(c + 0) * kHeadDim], v1 = src[(size_t)(c + 1) * kHeadDim];
-            const float v2 = src[(size_t)(c + 2) * kHeadDim], v3 = src[(size_t)(c + 3) * kHeadDim];
+        const float *src = po + (size_t)c0 * kHeadDim + d;
+        int c = g;
+        for (; c + 3 * kMergeGroups < n; c += 4 * kMergeGroups) {
+            const float v0 = src[(size_t)c * kHeadDim], v1 = src[(size_t)(c + kMergeGroups) * kHeadDim];
+            const float v2 = src[(size_t)(c + 2 * kMergeGroups) * kHeadDim], v3 = src[(size_t)(c + 3 * kMergeGroups) * kHeadDim];
             acc = fmaf(v0, w_s[c], acc);
-            acc = fmaf(v1, w_s[c + 1], acc);
-            acc = fmaf(v2, w_s[c + 2], acc);
-            acc = fmaf(v3, w_s[c + 3], acc);
+            acc = fmaf(v1, w_s[c + kMergeGroups], acc);
+            acc = fmaf(v2, w_s[c + 2 * kMergeGroups], acc);
+            acc = fmaf(v3, w_s[c + 3 * kMergeGroups], acc);
         }
-        for (; c < n; ++c) acc = fmaf(src[(size_t)c * kHeadDim], w_s[c], acc);
+        for (; c < n; c += kMergeGroups) acc = fmaf(src[(size_t)c * kHeadDim], w_s[c], acc);
     }
-    const float l = merge_block_reduce(lsum, false, red4, tid);
-    const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
-    out[(size_t)row * kHeadDim + tid] = __float2bfloat16_rn(acc * inv);
+    // ---- combine the four groups and the denominators (only the first 128 threads hold a share of lsum)
+    acc_s[g][d] = acc;
+    lsum = warp_sum(lsum);
+    __syncthreads();                       // red is free again (every thread has read the maxima)
+    if ((tid & 31) == 0) red[tid >> 5] = lsum;
+    __syncthreads();
+    if (g == 0) {
+        const float l = (red[0] + red[1]) + (red[2] + red[3]);   // the first four warps hold the shares
+        float o = acc_s[0][d];
+#pragma unroll
+        for (int i = 1; i < kMergeGroups; ++i) o += acc_s[i][d];
+        const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
+        out[(size_t)row * kHeadDim + d] = __float2bfloat16_rn(o * inv);
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -122,8 +132,13 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
     int C;
     const DecodeParams p = make_params(c, nullptr, kv_len, B, max_kv, Hq, 1.f, const_cast<void *>(workspace), C);
     const int rows = B * Hq;
-    SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel, dim3(rows), dim3(kMergeThreads), 0, stream, (const float *)p.part_o,
-                             (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
+    if (p.n_chunks >= 32) {
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, (const float *)p.part_o,
+                                 (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
+    } else {
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<1>, dim3(rows), dim3(kHeadDim), 0, stream, (const float *)p.part_o,
+                                 (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
+    }
     return SLIM_OK;
 }
 
