@@ -20,10 +20,11 @@
 //               other warp groups: setmaxnreg), then row maximum, exp2 -> fp16 P back to tensor memory and the
 //               running sum.  O is rescaled only when the maximum grows by more than 2^8.
 //
-// Scale bookkeeping: K^ = code * sk / kexp(j) with kexp(j) the power of two below the tile's largest K
-// scale, so s = acc * (kexp * row_scale); V^ = code * sv / vnorm with vnorm the power of two below the
-// largest V scale of the block's first key tile (one constant per block: the fp16 range absorbs the
-// variation between tiles), P = 2^(s - m), O = sum P . V^, l = sum P, out = O * vnorm / l.
+// Scale bookkeeping per key tile j: K^ = code * sk / kexp(j) and V^ = code * sv / vexp(j) with kexp(j), vexp(j)
+// the powers of two below the tile's largest K / V scale, so both operands stay in [0, 2) * 127 whatever the
+// magnitudes; s' = acc * (kexp * row_scale) + log2 vexp, P = 2^(s' - m), O += P . V^ (the factor vexp cancels
+// against 2^log2(vexp)), l += rowsum(P) / vexp, out = O / l.  vexp(j) is published as soon as the raw V tile has
+// landed (before its conversion), so the softmax of tile j never waits for it in practice.
 #include <cuda.h>
 
 #include "slim_common.cuh"
@@ -48,10 +49,12 @@ constexpr uint32_t kRaw = kVf + 32768;          // raw stages: 16 KB INT8 tile +
 constexpr uint32_t kRawStage = 17408;
 constexpr uint32_t kMisc = kRaw + kPfRawStages * kRawStage;
 constexpr uint32_t kBytes = kMisc + 512;
-// kMisc: floats [0,2) kexp of the K tile by parity of j, [2] vnorm, [4,16) converter warp maxima (3 x 4);
-//        byte 64: tensor-memory address; byte 72: failure flag; byte 128..: mbarriers
+// kMisc: floats by parity of the key tile j: [0,2) kexp, [2,4) log2 vexp, [12,14) 1 / vexp; converter warp maxima
+//        [4,12) for K tiles and [20,28) for V tiles; byte 64: tensor-memory address; byte 72: failure flag;
+//        byte 128..: mbarriers
 enum Bar { RAW_FULL = 0, RAW_EMPTY = kPfRawStages, KF_FULL = 2 * kPfRawStages, KF_EMPTY, VF_FULL, VF_EMPTY,
-           S_FULL, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, Q_FULL = O_DONE + 2, NUM_BARS = Q_FULL + 2 };
+           S_FULL, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, Q_FULL = O_DONE + 2, VEXP_FULL = Q_FULL + 2,
+           NUM_BARS = VEXP_FULL + 2 };
 static_assert(128 + 8 * NUM_BARS <= 512, "mbarriers fit the misc area");
 static_assert(kBytes <= 232448, "shared memory budget of one block");
 }  // namespace pfl
@@ -162,6 +165,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             tc::mbar_init(bar(pfl::P_FULL, t), 128);
             tc::mbar_init(bar(pfl::O_DONE, t), 1);
             tc::mbar_init(bar(pfl::Q_FULL, t), 128);
+            tc::mbar_init(bar(pfl::VEXP_FULL, t), 128);
         }
         tc::mbar_init_fence();
         *fail = 0;
@@ -242,7 +246,10 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             wait(bar(pfl::S_FULL, t), (uint32_t)j & 1u);
             __syncwarp();   // the wait loop may leave the lanes diverged; the tensor-memory ops below are warp-aligned
             tc::fence_after_sync();
+            wait(bar(pfl::VEXP_FULL, j & 1), (uint32_t)(j >> 1) & 1u);   // published long before, as a rule
             const float c = fmaxf(rs * misc_f[j & 1], 1e-37f);   // row scale * kexp of this key tile (> 0)
+            const float F = misc_f[2 + (j & 1)];                 // log2 vexp
+            const float vinv = misc_f[12 + (j & 1)];             // 1 / vexp
             const int key0 = j * kPfBN;
             const bool diag = key0 + kPfBN - 1 > last_key;       // some of this tile's keys are masked for this row
             // ---- the whole score row into registers with one round trip to tensor memory, then its maximum
@@ -272,7 +279,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 mx2 = pf_max3(mx2, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
             }
             mx = fmaxf(mx, mx2);
-            const float mt = (mx == -INFINITY) ? -INFINITY : mx * c;
+            const float mt = (mx == -INFINITY) ? -INFINITY : fmaf(mx, c, F);   // the tile's largest s'
             // the reference maximum only moves when the tile's exceeds it by more than the threshold
             const bool grow = (j == 0) ? true : (mt > m_run + kPfRescaleThreshold);
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
@@ -293,7 +300,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 l_run *= alpha;
             }
             if (grow) m_run = mt;
-            const float bias = (m_run == -INFINITY) ? 0.f : -m_run;
+            const float bias = (m_run == -INFINITY) ? 0.f : F - m_run;
             // ---- P = 2^(s - m) as fp16 pairs, packed in place, into the first 64 columns of the score buffer
             // (packed fp32 arithmetic: one fused multiply-add and one add per pair of scores)
             const uint64_t c2 = pf_pack(c, c), bias2 = pf_pack(bias, bias);
@@ -315,18 +322,18 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 tc::tmem_st32(tS, p0);
                 tc::tmem_st32(tS + 32, p1);
             }
-            l_run += rowsum;
+            l_run = fmaf(rowsum, vinv, l_run);
             tc::tmem_st_wait();
             tc::fence_before_sync();
             tc::mbar_arrive(bar(pfl::P_FULL, t));
         }
 
-        // ---- epilogue: O * vnorm / l -> bf16
+        // ---- epilogue: O / l -> bf16
         if (Tmine > 0) {
             wait(bar(pfl::O_DONE, t), (uint32_t)(Tmine - 1) & 1u);
             __syncwarp();
             tc::fence_after_sync();
-            const float inv_l = (l_run > 0.f) ? misc_f[2] / l_run : 0.f;
+            const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
             uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim);
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
@@ -356,31 +363,34 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     } else if (warp < 12) {
         // =========================================================== dequantise: thread = token row of the tile
         const int r = tid - 256, cw = warp - 8;
-        float *cmax = misc_f + 4;
-        float vnorm = 1.f;   // normalisation of the V operand, fixed by the first key tile
         for (int i = 0; i < 2 * T; ++i) {
             const int slot = i % kPfRawStages, j = i >> 1;
             const bool is_k = (i & 1) == 0;   // K tile first, then the V tile of the same keys
             wait(bar(pfl::RAW_FULL, slot), (uint32_t)(i / kPfRawStages) & 1u);
-            wait(bar(is_k ? pfl::KF_EMPTY : pfl::VF_EMPTY, 0), ((uint32_t)j & 1u) ^ 1u);
+            if (is_k) wait(bar(pfl::KF_EMPTY, 0), ((uint32_t)j & 1u) ^ 1u);
             const unsigned char *raw = smem + pfl::kRaw + slot * pfl::kRawStage;
             const int n_valid = min(kPfBN, kvl - j * kPfBN);   // rows past the cache length hold anything: zeroed
             const float sc = (r < n_valid) ? reinterpret_cast<const float *>(raw + 16384)[r] : 0.f;
-            float ex = vnorm;
-            if (is_k || j == 0) {
-                // power of two below the tile's largest scale (all K tiles; the V tile of the first keys);
-                // the exchange buffer alternates so that a fast warp cannot overwrite what a slow one still reads
-                float *cm = cmax + (is_k ? (j & 1) : 2) * 4;
-                const float wm = warp_max(sc);
-                if (lane == 0) cm[cw] = wm;
-                tc::named_barrier(1, 128);
-                const float tm = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
-                ex = (tm > 0.f) ? pow2_floor(tm) : 1.f;
-                if (!is_k) vnorm = ex;
-                if (r == 0) misc_f[is_k ? (j & 1) : 2] = ex;
+            // power of two below the tile's largest scale; the exchange buffers alternate with j so that a fast
+            // warp cannot overwrite what a slow one still reads
+            float *cm = misc_f + (is_k ? 4 : 20) + 4 * (j & 1);
+            const float wm = warp_max(sc);
+            if (lane == 0) cm[cw] = wm;
+            tc::named_barrier(1, 128);
+            const float tm = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
+            const float ex = (tm > 0.f) ? pow2_floor(tm) : 1.f;
+            if (is_k) {
+                if (r == 0) misc_f[j & 1] = ex;
+            } else {
+                // the softmax of this key tile needs the V exponent before the V tile itself is converted
+                if (r == 0) {
+                    misc_f[2 + (j & 1)] = (float)((int)(__float_as_uint(ex) >> 23) - 127);   // log2 of the power of two
+                    misc_f[12 + (j & 1)] = pow2_recip(ex);
+                }
+                tc::mbar_arrive(bar(pfl::VEXP_FULL, j & 1));
+                wait(bar(pfl::VF_EMPTY, 0), ((uint32_t)j & 1u) ^ 1u);
             }
-            // scale / 2^e: in [0, 2) for K; for V tiles beyond the first kept finite in fp16 (code * factor < 65504)
-            const float f = fminf(sc * pow2_recip(ex), 256.f);
+            const float f = sc * pow2_recip(ex);   // scale / 2^e in [0, 2)
             const uint32_t fac2 = pack_half2(f, f);
             unsigned char *dstb = smem + (is_k ? pfl::kKf : pfl::kVf) + r * 128;
 #pragma unroll

@@ -255,3 +255,23 @@ def test_decode_step_from_host_buffers():
     for b in range(B):
         want = so.attention(bf16_bits(w.q_decode[0, b:b + 1]), *oc[b], ctx[b] + 1, w.sm_scale)
         _assert_close(out[b:b + 1], want, f"host step seq {b}")
+
+
+def test_prefill_scale_jumps_between_key_tiles():
+    # K and V magnitudes that differ by 2^18 from one 128-key tile to the next, in both directions: every key tile
+    # is normalised by its own power of two, so none of them may overflow or vanish in the fp16 operands
+    w = _custom(1, 2, 1, [512], [0], 0, 800)
+    w.v[0][0:128] *= 2.0 ** -12
+    w.v[0][128:256] *= 2.0 ** 6
+    w.v[0][384:512] *= 2.0 ** -3
+    w.k[0][256:384] *= 2.0 ** -10
+    w.k[0][384:512] *= 2.0 ** 3
+    oc = _oracle_cache(w)
+    from paper_2407_07304_b200 import harness
+    run, out_prefill, _ = harness.run_workload(w)
+    _assert_cache_bits(run, oc)
+    want = so.attention(bf16_bits(w.q_prefill[0]), *oc[0], 512, w.sm_scale)
+    got = out_prefill[0].float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    denom = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
+    assert (np.abs(got - want) / denom).max() < 2e-2
