@@ -231,6 +231,14 @@ int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
  */
 int slim_read_status(const void *workspace, void *stream);
 
+/*
+ * Exercises that failure path without any failure: launches one thread that waits, with the kernels' bounded
+ * wait and a short limit, on a barrier nothing arrives on; the wait runs out, the thread stores
+ * SLIM_ERR_TIMEOUT in the first word of `workspace` (device, 4-byte aligned) and the kernel ends normally.
+ * slim_read_status(workspace) then returns SLIM_ERR_TIMEOUT; the CUDA context stays usable.
+ */
+int slim_selftest_timeout(void *workspace, void *stream);
+
 /* Scratch bytes needed by a phase (SLIM_PHASE_*) for the given shape; 0 on invalid arguments. */
 size_t slim_workspace_bytes(int32_t phase, int32_t B, int32_t Hq, int32_t Hkv, int32_t max_q, int32_t max_kv);
 

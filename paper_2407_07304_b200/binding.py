@@ -25,7 +25,7 @@ PAGE_TOKENS = 128
 
 EXPORTS = (
     "slim_kv_append", "slim_attn_prefill", "slim_attn_decode", "slim_attn_decode_split",
-    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_workspace_bytes",
+    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -86,6 +86,8 @@ def lib():
         L.slim_step_staging_bytes.restype = Z
         L.slim_read_status.argtypes = [P, P]
         L.slim_read_status.restype = ctypes.c_int
+        L.slim_selftest_timeout.argtypes = [P, P]
+        L.slim_selftest_timeout.restype = ctypes.c_int
         L.slim_workspace_bytes.argtypes = [I, I, I, I, I, I]
         L.slim_workspace_bytes.restype = Z
         L.slim_cache_code_bytes.argtypes = [I, I]
@@ -207,6 +209,11 @@ def slim_decode_step_host(cache, q_host, k_new_host, v_new_host, out_host, stagi
 def slim_read_status(workspace, stream=None):
     """Synchronises the stream and returns SLIM_OK or SLIM_ERR_TIMEOUT (a bounded device-side wait ran out)."""
     return lib().slim_read_status(_ptr(workspace), _stream(stream))
+
+
+def slim_selftest_timeout(workspace, stream=None):
+    """Makes a bounded device-side wait run out on purpose (nothing faults); the status word of `workspace` is set."""
+    _check(lib().slim_selftest_timeout(_ptr(workspace), _stream(stream)), "slim_selftest_timeout")
 
 
 def slim_step_staging_bytes(B, Hq, Hkv):

@@ -1,5 +1,6 @@
 // C ABI of the library (declared in include/slim.h): argument validation and dispatch.
 #include "slim_common.cuh"
+#include "slim_tcgen05.cuh"
 
 #define SLIM_EXPORT extern "C" __attribute__((visibility("default")))
 
@@ -178,6 +179,25 @@ SLIM_EXPORT int slim_read_status(const void *workspace, void *stream)
     SLIM_CUDA_TRY(cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     SLIM_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return (word == 0) ? SLIM_OK : SLIM_ERR_TIMEOUT;
+}
+
+// One thread waits on an mbarrier that nothing ever arrives on, with the same bounded wait the attention kernels
+// use (a short limit here), and reports the way they do: SLIM_ERR_TIMEOUT in the status word, normal exit.
+__global__ void slim_selftest_timeout_kernel(int *status)
+{
+    __shared__ __align__(8) unsigned long long mbar;
+    const uint32_t addr = slim::smem_u32(&mbar);
+    slim::tc::mbar_init(addr, 1);
+    slim::tc::mbar_init_fence();
+    if (!slim::tc::mbar_wait(addr, 0, 64u)) atomicExch(status, SLIM_ERR_TIMEOUT);
+}
+
+SLIM_EXPORT int slim_selftest_timeout(void *workspace, void *stream)
+{
+    if (workspace == nullptr || ((uintptr_t)workspace & 3)) return SLIM_ERR_INVALID_ARG;
+    slim_selftest_timeout_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(static_cast<int *>(workspace));
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
 }
 
 SLIM_EXPORT size_t slim_cache_code_bytes(int32_t num_pages, int32_t num_kv_heads)

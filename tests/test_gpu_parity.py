@@ -275,3 +275,16 @@ def test_prefill_scale_jumps_between_key_tiles():
     assert np.isfinite(got).all()
     denom = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
     assert (np.abs(got - want) / denom).max() < 2e-2
+
+
+def test_a_wait_that_runs_out_is_reported_not_hung():
+    # the failure path of the bounded waits, exercised without any failure: a barrier nothing arrives on
+    from paper_2407_07304_b200 import binding as slim, harness
+    ws = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    assert slim.slim_read_status(ws) == slim.SLIM_OK
+    slim.slim_selftest_timeout(ws)
+    assert slim.slim_read_status(ws) == slim.SLIM_ERR_TIMEOUT
+    ws.zero_()
+    assert slim.slim_read_status(ws) == slim.SLIM_OK
+    # the context is intact: a normal run still matches the oracle
+    _check(_custom(1, 2, 1, [40], [0], 1, 900))
