@@ -263,7 +263,11 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.synchronize()
     split_ms = [a.elapsed_time(b) for a, b in evs]
     # ---- end to end: host (pinned) inputs and outputs through slim_decode_step_host
-    q_h, k_h, v_h = q.cpu().pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+    # one pinned allocation holding q | k_new | v_new back to back: the step copies it with one transfer
+    n_q, n_kv = q.numel(), k_new.numel()
+    host_in = torch.empty(n_q + 2 * n_kv, dtype=torch.bfloat16).pin_memory()
+    q_h, k_h, v_h = host_in[:n_q].view_as(q), host_in[n_q:n_q + n_kv].view_as(k_new), host_in[n_q + n_kv:].view_as(v_new)
+    q_h.copy_(q.cpu()), k_h.copy_(k_new.cpu()), v_h.copy_(v_new.cpu())
     out_h = torch.empty_like(q_h).pin_memory()
     staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
 

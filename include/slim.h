@@ -168,6 +168,9 @@ int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
  * cache traffic Eq. 1 counts).  Host buffers should be pinned; they must stay
  * valid and out_host must not be read until the stream has been synchronised.
  *
+ * If q_host, k_new_host and v_new_host lie back to back in one allocation (in that order) they are copied with
+ * one transfer instead of three.
+ *
  *   q_host      host bf16 [B][Hq][128]
  *   k_new_host, v_new_host  host bf16 [B][num_kv_heads][128]
  *   out_host    host bf16 [B][Hq][128]

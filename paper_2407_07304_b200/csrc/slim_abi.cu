@@ -150,9 +150,16 @@ SLIM_EXPORT int slim_decode_step_host(const slim_cache_t *cache, const void *q_h
     cudaStream_t st = (cudaStream_t)stream;
     const size_t q_bytes = (size_t)B * Hq * SLIM_HEAD_DIM * 2, kv_bytes = (size_t)B * Hkv * SLIM_HEAD_DIM * 2;
     char *d_q = static_cast<char *>(staging), *d_k = d_q + q_bytes, *d_v = d_k + kv_bytes, *d_o = d_v + kv_bytes;
-    SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
-    SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, k_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
-    SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, v_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    const char *hq = static_cast<const char *>(q_host), *hk = static_cast<const char *>(k_new_host),
+               *hv = static_cast<const char *>(v_new_host);
+    if (hk == hq + q_bytes && hv == hk + kv_bytes) {
+        // the three host buffers are adjacent (one allocation): one copy instead of three
+        SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, hq, q_bytes + 2 * kv_bytes, cudaMemcpyHostToDevice, st));
+    } else {
+        SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, hq, q_bytes, cudaMemcpyHostToDevice, st));
+        SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, hk, kv_bytes, cudaMemcpyHostToDevice, st));
+        SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, hv, kv_bytes, cudaMemcpyHostToDevice, st));
+    }
     rc = launch_append(cache, d_k, d_v, cu_new, start_pos, B, 1, st);
     if (rc != SLIM_OK) return rc;
     rc = launch_decode_split(cache, d_q, kv_len, B, max_kv, Hq, sm_scale, workspace, st);

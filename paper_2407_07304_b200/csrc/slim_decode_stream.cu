@@ -653,11 +653,13 @@ int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int
     const unsigned grid = (unsigned)(max_items < sms ? max_items : sms);
     if (p.G <= 8) {
         constexpr int bytes = (int)StSmem<8>::kBytes;
-        SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<8>), bytes);
+        if (rc != SLIM_OK) return rc;
         SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<8>, dim3(grid), dim3(StSmem<8>::kThreads), bytes, stream, map_tile, map_tail, p, B));
     } else {
         constexpr int bytes = (int)StSmem<16>::kBytes;
-        SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_decode_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+        rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<16>), bytes);
+        if (rc != SLIM_OK) return rc;
         SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<16>, dim3(grid), dim3(StSmem<16>::kThreads), bytes, stream, map_tile, map_tail, p, B));
     }
     SLIM_CUDA_TRY(cudaGetLastError());

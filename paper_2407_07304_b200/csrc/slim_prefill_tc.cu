@@ -540,7 +540,8 @@ int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int
     CUtensorMap map;
     int rc = codes_tensor_map(c, kPfBN, &map);
     if (rc != SLIM_OK) return rc;
-    SLIM_CUDA_TRY(cudaFuncSetAttribute(slim_prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pfl::kBytes));
+    rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_prefill_tc_kernel), (int)pfl::kBytes);
+    if (rc != SLIM_OK) return rc;
     dim3 grid((unsigned)p.n_qblocks, (unsigned)Hq, (unsigned)B);
     slim_prefill_tc_kernel<<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
     SLIM_CUDA_TRY(cudaGetLastError());

@@ -82,4 +82,23 @@ int sm_count(int *out)
     return SLIM_OK;
 }
 
+int allow_dynamic_smem(const void *func, int bytes)
+{
+    struct Done {
+        int dev;
+        const void *func;
+    };
+    static std::mutex mu;
+    static Done done[64];
+    static int n_done = 0;
+    int dev = 0;
+    SLIM_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < n_done; ++i)
+        if (done[i].dev == dev && done[i].func == func) return SLIM_OK;
+    SLIM_CUDA_TRY(cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    if (n_done < 64) done[n_done++] = Done{dev, func};
+    return SLIM_OK;
+}
+
 }  // namespace slim

@@ -13,4 +13,8 @@ int codes_tensor_map(const slim_cache_t *c, int box_rows, CUtensorMap *out);
 // Number of SMs of the current device (cached per device).
 int sm_count(int *out);
 
+// cudaFuncSetAttribute(func, MaxDynamicSharedMemorySize, bytes), issued once per (device, kernel) instead of on
+// every launch; thread-safe.
+int allow_dynamic_smem(const void *func, int bytes);
+
 }  // namespace slim
