@@ -279,9 +279,38 @@ def run_ours(args, rank, world, local_rank):
 
     for i in range(3):
         step_host(i)
-    ms_e2e = timed(step_host, args.steps)
-    clocks = sampler.stop() if sampler else None
+    ms_e2e_eager = timed(step_host, args.steps)
     same = torch.equal(out_h, out.cpu())
+    # The same call captured once per cache copy into a CUDA graph (copy in, three kernels, copy out) and replayed:
+    # what a serving loop does with a fixed-shape decode step.  The graph reads the pinned buffers at replay time.
+    side = torch.cuda.Stream()
+    graphs = []
+    with torch.cuda.stream(side):
+        for i in range(N_ROT):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+                slim.slim_decode_step_host(runs[i].cache, q_h, k_h, v_h, out_h, staging, cu_new, start_pos, kv_len, B,
+                                           max_kv, Hq, w.sm_scale, ws, side)
+            graphs.append(g)
+        out_h.zero_()
+
+        def step_graph(i):
+            graphs[i % N_ROT].replay()
+            side.synchronize()      # the caller needs the result before the next token
+
+        for i in range(3):
+            step_graph(i)
+        same = same and torch.equal(out_h, out.cpu())
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for i in range(args.steps):
+            step_graph(i)
+        e1.record(side)
+        torch.cuda.synchronize()
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        barrier()
+    clocks = sampler.stop() if sampler else None
 
     # ---- extra single-GPU context numbers (not part of the headline): prefill of workload 3
     extra = {}
@@ -316,7 +345,9 @@ def run_ours(args, rank, world, local_rank):
                      "frac_of_8tbs": achieved / 8000.0, "bytes_per_launch": split_bytes,
                      "avg_launch_ms": split_avg_ms, "min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
         "e2e": {"value": whole_job_rate(B, args.steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same)},
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same),
+                "launch": "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step",
+                "ms_per_step_without_graph": ms_e2e_eager / args.steps},
         "gpu_launches": 3 * args.steps,
         "clocks": clocks,
     }

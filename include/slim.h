@@ -171,6 +171,10 @@ int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
  * If q_host, k_new_host and v_new_host lie back to back in one allocation (in that order) they are copied with
  * one transfer instead of three.
  *
+ * The call synchronises nothing and allocates nothing.  After one ordinary call with the same cache and shapes
+ * (which creates the tensor map and sets the kernels' attributes) it may be recorded by stream capture into a
+ * CUDA graph; the graph reads the host buffers when it is replayed.
+ *
  *   q_host      host bf16 [B][Hq][128]
  *   k_new_host, v_new_host  host bf16 [B][num_kv_heads][128]
  *   out_host    host bf16 [B][Hq][128]
