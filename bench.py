@@ -217,17 +217,15 @@ def run_ours(args, rank, world, local_rank):
     v_new = torch.cat([w.v[b][ctx:ctx + 1] for b in range(B)]).to(dev).contiguous()
     q = w.q_decode[0].to(dev).contiguous()
     out = torch.empty_like(q)
-    cu_new = torch.arange(B + 1, dtype=torch.int32, device=dev)
-    start_pos = torch.full((B,), ctx, dtype=torch.int32, device=dev)
     kv_len = torch.full((B,), ctx + 1, dtype=torch.int32, device=dev)
     max_kv = ctx + 1
     ws = runs[0].ws_decode
     stream = torch.cuda.current_stream()
 
     def step(i):
-        c = runs[i % N_ROT].cache
-        slim.slim_kv_append(c, k_new, v_new, cu_new, start_pos, B, 1, stream)
-        slim.slim_attn_decode(c, q, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
+        # one call, two kernels: the split kernel quantises the new token's K/V rows into the cache before it reads
+        # them, the merge kernel combines the partial results
+        slim.slim_decode_step(runs[i % N_ROT].cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
 
     def timed(fn, steps):
         barrier()
@@ -249,15 +247,13 @@ def run_ours(args, rank, world, local_rank):
         time.sleep(0.1)
     # ---- headline: device-resident inputs, whole step
     ms_total = timed(step, args.steps)
-    # ---- per-kernel: the split kernel alone, events around every launch
-    split_ms = []
+    # ---- per-kernel: the step's split kernel (new rows written, cache streamed) alone, events around every launch
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     barrier()
     for i in range(args.steps):
         c = runs[i % N_ROT].cache
-        slim.slim_kv_append(c, k_new, v_new, cu_new, start_pos, B, 1, stream)
         evs[i][0].record(stream)
-        slim.slim_attn_decode_split(c, q, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
+        slim.slim_attn_decode_split(c, q, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream, k_new=k_new, v_new=v_new)
         evs[i][1].record(stream)
         slim.slim_attn_decode_merge(c, out, kv_len, B, max_kv, Hq, ws, stream)
     torch.cuda.synchronize()
@@ -273,8 +269,7 @@ def run_ours(args, rank, world, local_rank):
 
     def step_host(i):
         c = runs[i % N_ROT].cache
-        slim.slim_decode_step_host(c, q_h, k_h, v_h, out_h, staging, cu_new, start_pos, kv_len, B, max_kv, Hq,
-                                   w.sm_scale, ws, stream)
+        slim.slim_decode_step_host(c, q_h, k_h, v_h, out_h, staging, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
         stream.synchronize()        # the caller needs the result before the next token
 
     for i in range(3):
@@ -289,8 +284,8 @@ def run_ours(args, rank, world, local_rank):
         for i in range(N_ROT):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
-                slim.slim_decode_step_host(runs[i].cache, q_h, k_h, v_h, out_h, staging, cu_new, start_pos, kv_len, B,
-                                           max_kv, Hq, w.sm_scale, ws, side)
+                slim.slim_decode_step_host(runs[i].cache, q_h, k_h, v_h, out_h, staging, kv_len, B, max_kv, Hq,
+                                           w.sm_scale, ws, side)
             graphs.append(g)
         out_h.zero_()
 
@@ -322,9 +317,9 @@ def run_ours(args, rank, world, local_rank):
     hbm_peak, bf16_peak, peak_kind = _peaks()
     tokens = world * B * args.steps
     cache_bytes = sum(kv_len_host) * Hkv * ROW_BYTES
-    split_bytes = cache_bytes + B * Hq * 128 * 2
     # whole step: cache read once, Q in, O out, new K/V rows read as bf16 and written as codes + scales
     step_bytes = cache_bytes + 2 * B * Hq * 256 + B * Hkv * (2 * 256 + ROW_BYTES)
+    split_bytes = step_bytes - B * Hq * 256      # the split kernel: all of that but the final output
     split_avg_ms = statistics.mean(split_ms)
     achieved = split_bytes / (split_avg_ms * 1e-3) / 1e9
     h2d = (B * Hq + 2 * B * Hkv) * 128 * 2
@@ -348,7 +343,7 @@ def run_ours(args, rank, world, local_rank):
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same),
                 "launch": "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step",
                 "ms_per_step_without_graph": ms_e2e_eager / args.steps},
-        "gpu_launches": 3 * args.steps,
+        "gpu_launches": 2 * args.steps,
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu:
@@ -360,9 +355,9 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
-# dram bytes read + written by one slim_decode_stream_kernel launch on this workload (279.68 MB read,
-# 6.07 MB written), from the ncu capture summarised under profiles/.
-TRAFFIC_PER_LAUNCH = 285.75e6
+# dram bytes read + written by one slim_decode_stream_kernel launch on this workload, from the ncu capture
+# summarised under profiles/; None while the kernel is newer than the last capture.
+TRAFFIC_PER_LAUNCH = None
 
 
 def extra_numbers(slim, workloads, dev):

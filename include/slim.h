@@ -151,9 +151,13 @@ int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out,
  * chunk, one softmax over the chunk, the product with V; Section 2.1 order inside
  * the chunk) writes partials into `workspace`; the merge pass combines them into
  * `out`.  Same arguments, validation and workspace as slim_attn_decode;
- * slim_attn_decode(...) == split(...) followed by merge(...) on the same stream.
+ * slim_attn_decode(...) == split(..., NULL, NULL, ...) followed by merge(...) on
+ * the same stream.  With k_new and v_new (both or neither; as for
+ * slim_decode_step) the split pass first writes every sequence's new token into
+ * slot kv_len[b] - 1: slim_decode_step(...) == split(..., k_new, v_new, ...)
+ * followed by merge(...).
  */
-int slim_attn_decode_split(const slim_cache_t *cache, const void *q,
+int slim_attn_decode_split(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new,
                            const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
                            void *workspace, size_t workspace_bytes, void *stream);
 int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
@@ -161,11 +165,30 @@ int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
                            const void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * One decode step in one call: the new token of every sequence is quantised into
+ * the cache (exactly as slim_kv_append does, Section 2.2) at position
+ * kv_len[b] - 1 and decode attention runs over all kv_len[b] tokens, the new one
+ * included; the result equals slim_kv_append(start_pos = kv_len - 1) followed by
+ * slim_attn_decode, bit for bit.  The quantisation happens inside the split
+ * kernel of the attention (the thread block that reads a sequence's last key
+ * chunk writes the new row first), so the step has no separate append kernel.
+ *
+ *   k_new, v_new  device bf16 [B][num_kv_heads][128], 16-byte aligned
+ *   kv_len        device int32 [B]: cached tokens per sequence counting the new
+ *                 one; a sequence with kv_len[b] <= 0 appends nothing and gets
+ *                 zeros; a kv_len[b] beyond max_kv or the page table appends
+ *                 nothing and attends over the tokens that fit
+ *   others        as for slim_attn_decode
+ */
+int slim_decode_step(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new, void *out,
+                     const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * One decode step from host buffers: copies the step's query and new K/V rows
- * (one new token per sequence) host -> device, appends them (slim_kv_append),
- * runs slim_attn_decode over the lengthened cache and copies the result device
- * -> host, all asynchronously on `stream` (Section 2.2: the per-token step whose
- * cache traffic Eq. 1 counts).  Host buffers should be pinned; they must stay
+ * (one new token per sequence) host -> device, runs slim_decode_step and copies
+ * the result device -> host, all asynchronously on `stream` (Section 2.2: the
+ * per-token step whose cache traffic Eq. 1 counts).  Host buffers should be pinned; they must stay
  * valid and out_host must not be read until the stream has been synchronised.
  *
  * If q_host, k_new_host and v_new_host lie back to back in one allocation (in that order) they are copied with
@@ -179,15 +202,12 @@ int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
  *   k_new_host, v_new_host  host bf16 [B][num_kv_heads][128]
  *   out_host    host bf16 [B][Hq][128]
  *   staging     device scratch of at least slim_step_staging_bytes(B, Hq, Hkv) bytes, 16-byte aligned
- *   cu_new      device int32 [B+1] = 0, 1, ..., B
- *   start_pos   device int32 [B]: position the new token of sequence b is written to
- *   kv_len      device int32 [B]: cached tokens per sequence after the append (start_pos + 1)
+ *   kv_len      device int32 [B]: cached tokens per sequence counting the new one
  *   workspace   as for slim_attn_decode
  */
 int slim_decode_step_host(const slim_cache_t *cache, const void *q_host, const void *k_new_host,
                           const void *v_new_host, void *out_host, void *staging, size_t staging_bytes,
-                          const int32_t *cu_new, const int32_t *start_pos, const int32_t *kv_len,
-                          int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                          const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
                           void *workspace, size_t workspace_bytes, void *stream);
 size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
 

@@ -25,7 +25,7 @@ PAGE_TOKENS = 128
 
 EXPORTS = (
     "slim_kv_append", "slim_attn_prefill", "slim_attn_decode", "slim_attn_decode_split",
-    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
+    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -74,13 +74,15 @@ def lib():
         L.slim_attn_prefill.restype = ctypes.c_int
         L.slim_attn_decode.argtypes = [CP, P, P, P, I, I, I, F, P, Z, P]
         L.slim_attn_decode.restype = ctypes.c_int
-        L.slim_attn_decode_split.argtypes = [CP, P, P, I, I, I, F, P, Z, P]
+        L.slim_attn_decode_split.argtypes = [CP, P, P, P, P, I, I, I, F, P, Z, P]
         L.slim_attn_decode_split.restype = ctypes.c_int
         L.slim_attn_decode_merge.argtypes = [CP, P, P, I, I, I, P, Z, P]
         L.slim_attn_decode_merge.restype = ctypes.c_int
         L.slim_attn_decode_static.argtypes = [CP, P, P, P, I, I, I, F, P]
         L.slim_attn_decode_static.restype = ctypes.c_int
-        L.slim_decode_step_host.argtypes = [CP, P, P, P, P, P, Z, P, P, P, I, I, I, F, P, Z, P]
+        L.slim_decode_step.argtypes = [CP, P, P, P, P, P, I, I, I, F, P, Z, P]
+        L.slim_decode_step.restype = ctypes.c_int
+        L.slim_decode_step_host.argtypes = [CP, P, P, P, P, P, Z, P, I, I, I, F, P, Z, P]
         L.slim_decode_step_host.restype = ctypes.c_int
         L.slim_step_staging_bytes.argtypes = [I, I, I]
         L.slim_step_staging_bytes.restype = Z
@@ -172,9 +174,9 @@ def slim_attn_decode(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, workspace, 
     _check(rc, "slim_attn_decode")
 
 
-def slim_attn_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None):
-    rc = lib().slim_attn_decode_split(ctypes.byref(cache.struct), _ptr(q), _ptr(kv_len), B, max_kv, Hq, sm_scale,
-                                      _ptr(workspace), _nbytes(workspace), _stream(stream))
+def slim_attn_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None, k_new=None, v_new=None):
+    rc = lib().slim_attn_decode_split(ctypes.byref(cache.struct), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(kv_len), B, max_kv,
+                                      Hq, sm_scale, _ptr(workspace), _nbytes(workspace), _stream(stream))
     _check(rc, "slim_attn_decode_split")
 
 
@@ -196,13 +198,19 @@ def slim_attn_decode_static(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, stre
     _check(rc, "slim_attn_decode_static")
 
 
-def slim_decode_step_host(cache, q_host, k_new_host, v_new_host, out_host, staging, cu_new, start_pos, kv_len,
-                          B, max_kv, Hq, sm_scale, workspace, stream=None):
+def slim_decode_step(cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None):
+    """Appends one token per sequence at position kv_len - 1 and attends over kv_len tokens, in one kernel."""
+    rc = lib().slim_decode_step(ctypes.byref(cache.struct), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(kv_len),
+                                B, max_kv, Hq, sm_scale, _ptr(workspace), _nbytes(workspace), _stream(stream))
+    _check(rc, "slim_decode_step")
+
+
+def slim_decode_step_host(cache, q_host, k_new_host, v_new_host, out_host, staging, kv_len, B, max_kv, Hq, sm_scale,
+                          workspace, stream=None):
     """q_host / k_new_host / v_new_host / out_host are CPU (pinned) bf16 tensors."""
     rc = lib().slim_decode_step_host(ctypes.byref(cache.struct), _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host),
-                                     _ptr(out_host), _ptr(staging), _nbytes(staging), _ptr(cu_new), _ptr(start_pos),
-                                     _ptr(kv_len), B, max_kv, Hq, sm_scale, _ptr(workspace), _nbytes(workspace),
-                                     _stream(stream))
+                                     _ptr(out_host), _ptr(staging), _nbytes(staging), _ptr(kv_len), B, max_kv, Hq,
+                                     sm_scale, _ptr(workspace), _nbytes(workspace), _stream(stream))
     _check(rc, "slim_decode_step_host")
 
 

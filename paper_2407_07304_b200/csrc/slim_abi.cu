@@ -16,10 +16,12 @@ int set_cuda_error(cudaError_t e)
 
 int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
                   const int32_t *start_pos, int B, int max_new, cudaStream_t stream);
-int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv, int Hq,
-                        float sm_scale, void *workspace, cudaStream_t stream);
+int launch_decode_split(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, const int32_t *kv_len,
+                        int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
                         const void *workspace, cudaStream_t stream);
+int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, void *out,
+                  const int32_t *kv_len, int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                       int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
@@ -90,15 +92,16 @@ static int check_decode(const slim_cache_t *cache, int32_t B, int32_t max_kv, in
     return SLIM_OK;
 }
 
-SLIM_EXPORT int slim_attn_decode_split(const slim_cache_t *cache, const void *q, const int32_t *kv_len, int32_t B,
-                                       int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
-                                       size_t workspace_bytes, void *stream)
+SLIM_EXPORT int slim_attn_decode_split(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new,
+                                       const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                                       void *workspace, size_t workspace_bytes, void *stream)
 {
     bool launch;
     int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
     if (rc != SLIM_OK || !launch) return rc;
     if (q == nullptr || kv_len == nullptr || ((uintptr_t)q & 15)) return SLIM_ERR_INVALID_ARG;
-    return launch_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+    if ((k_new == nullptr) != (v_new == nullptr) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15)) return SLIM_ERR_INVALID_ARG;
+    return launch_decode_split(cache, q, k_new, v_new, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
 }
 
 SLIM_EXPORT int slim_attn_decode_merge(const slim_cache_t *cache, void *out, const int32_t *kv_len, int32_t B,
@@ -121,9 +124,20 @@ SLIM_EXPORT int slim_attn_decode(const slim_cache_t *cache, const void *q, void 
     if (rc != SLIM_OK || !launch) return rc;
     if (q == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
     if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
-    rc = launch_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
-    if (rc != SLIM_OK) return rc;
-    return launch_decode_merge(cache, out, kv_len, B, max_kv, Hq, workspace, (cudaStream_t)stream);
+    return launch_decode(cache, q, nullptr, nullptr, out, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_decode_step(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new, void *out,
+                                 const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                                 void *workspace, size_t workspace_bytes, void *stream)
+{
+    bool launch;
+    int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (q == nullptr || k_new == nullptr || v_new == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15))
+        return SLIM_ERR_INVALID_ARG;
+    return launch_decode(cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
 }
 
 SLIM_EXPORT size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv)
@@ -134,15 +148,13 @@ SLIM_EXPORT size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv)
 
 SLIM_EXPORT int slim_decode_step_host(const slim_cache_t *cache, const void *q_host, const void *k_new_host,
                                       const void *v_new_host, void *out_host, void *staging, size_t staging_bytes,
-                                      const int32_t *cu_new, const int32_t *start_pos, const int32_t *kv_len,
-                                      int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
+                                      const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
                                       size_t workspace_bytes, void *stream)
 {
     bool launch;
     int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
     if (rc != SLIM_OK || !launch) return rc;
-    if (q_host == nullptr || k_new_host == nullptr || v_new_host == nullptr || out_host == nullptr ||
-        cu_new == nullptr || start_pos == nullptr || kv_len == nullptr)
+    if (q_host == nullptr || k_new_host == nullptr || v_new_host == nullptr || out_host == nullptr || kv_len == nullptr)
         return SLIM_ERR_INVALID_ARG;
     const int Hkv = cache->num_kv_heads;
     if (staging == nullptr || ((uintptr_t)staging & 15) || staging_bytes < slim_step_staging_bytes(B, Hq, Hkv))
@@ -160,11 +172,7 @@ SLIM_EXPORT int slim_decode_step_host(const slim_cache_t *cache, const void *q_h
         SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, hk, kv_bytes, cudaMemcpyHostToDevice, st));
         SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, hv, kv_bytes, cudaMemcpyHostToDevice, st));
     }
-    rc = launch_append(cache, d_k, d_v, cu_new, start_pos, B, 1, st);
-    if (rc != SLIM_OK) return rc;
-    rc = launch_decode_split(cache, d_q, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
-    if (rc != SLIM_OK) return rc;
-    rc = launch_decode_merge(cache, d_o, kv_len, B, max_kv, Hq, workspace, st);
+    rc = launch_decode(cache, d_q, d_k, d_v, d_o, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
     if (rc != SLIM_OK) return rc;
     SLIM_CUDA_TRY(cudaMemcpyAsync(out_host, d_o, q_bytes, cudaMemcpyDeviceToHost, st));
     return SLIM_OK;

@@ -114,16 +114,32 @@ static DecodeParams make_params(const slim_cache_t *c, const void *q, const int3
     p.status = static_cast<int *>(workspace);
     p.part_o = reinterpret_cast<float *>(static_cast<char *>(workspace) + kDecodeStatusBytes);
     p.part_ml = p.part_o + (size_t)B * Hq * p.n_chunks * kHeadDim;
+    p.k_new = p.v_new = nullptr;
     return p;
 }
 
-int launch_decode_split(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv, int Hq,
-                        float sm_scale, void *workspace, cudaStream_t stream)
+int launch_decode_split(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, const int32_t *kv_len,
+                        int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream)
 {
     int C;
-    const DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
+    DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
     if (p.n_chunks == 0) return SLIM_OK;
+    p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
     return launch_decode_split_stream(c, p, B, stream);
+}
+
+int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
+                        const void *workspace, cudaStream_t stream);
+
+// Decode attention: split kernel, then merge kernel.  With k_new / v_new the split kernel first quantises every
+// sequence's new token into slot kv_len - 1 of the cache (the one-call decode step).
+int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, void *out,
+                  const int32_t *kv_len, int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream)
+{
+    const int rc = launch_decode_split(c, q, k_new, v_new, kv_len, B, max_kv, Hq, sm_scale, workspace, stream);
+    if (rc != SLIM_OK) return rc;
+    return launch_decode_merge(c, out, kv_len, B, max_kv, Hq, workspace, stream);
 }
 
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
@@ -197,8 +213,6 @@ int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
     void *scratch = nullptr;
     int rc = static_scratch_address(&scratch);
     if (rc != SLIM_OK) return rc;
-    rc = launch_decode_split(cache, q, kv_len, B, max_kv, Hq, sm_scale, scratch, (cudaStream_t)stream);
-    if (rc != SLIM_OK) return rc;
-    return launch_decode_merge(cache, out, kv_len, B, max_kv, Hq, scratch, (cudaStream_t)stream);
+    return launch_decode(cache, q, nullptr, nullptr, out, kv_len, B, max_kv, Hq, sm_scale, scratch, (cudaStream_t)stream);
 }
 

@@ -13,6 +13,9 @@ struct DecodeParams {
     int *status;              // first word of the workspace: set to a SLIM_ERR_* code by a kernel whose wait ran out
     float *part_o;            // [B][Hq][n_chunks][128] unnormalised partial outputs
     float *part_ml;           // [B][Hq][n_chunks][2]   (max in log2 units, sum)
+    // one-kernel append + split (optional): the new token of every sequence, [B][Hkv][128], quantised into slot
+    // kv_len - 1 by the block that owns the sequence's last chunk (null: nothing to append)
+    const __nv_bfloat16 *k_new, *v_new;
     int Hq, Hkv, G;
     int max_pages_per_seq, num_pages, n_chunks;
     float scale_log2e;        // sm_scale * log2(e)

@@ -36,6 +36,7 @@
 
 #include "slim_common.cuh"
 #include "slim_decode_params.cuh"
+#include "slim_quant.cuh"
 #include "slim_tcgen05.cuh"
 #include "slim_tmap.cuh"
 
@@ -51,7 +52,7 @@ constexpr float kStPFix = 65535.f;
 
 static_assert(kStChunk == 256, "partials are indexed by 256-token chunks (decode_workspace_bytes, merge kernel)");
 
-template <int NH>
+template <int NH, bool kAppend = false>
 struct StSmem {
     static constexpr int N = 2 * NH;                        // MMA columns: [hi bytes of NH heads | lo bytes]
     static constexpr int kGroups = (NH <= 8) ? 3 : 2;       // consumer groups (chunks in process at a time)
@@ -79,8 +80,9 @@ struct StSmem {
     static constexpr uint32_t kBar = kGroup0 + kGroups * kGroupBytes;
     static constexpr int kNumBars = 2 * kStages + 2 * kInfoSlots + 4 * kGroups;
     static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
-    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[4]: chunks of this block, first sequence / head / chunk
-    static constexpr uint32_t kFail = kRange + 16;
+    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[5]: chunks of this block, first sequence / head / chunk, that sequence's chunks
+    static constexpr uint32_t kFail = kRange + 32;
+    static constexpr uint32_t kAppended = kFail + 4;       // int: consumer warps that have written their share of the new-token rows
     static constexpr uint32_t kBytes = kFail + 8;
     static_assert(kRange % 16 == 0, "range record is read as int4-aligned ints");
     static_assert(kBytes <= 232448, "shared memory budget of one block");
@@ -124,12 +126,38 @@ __device__ __forceinline__ int st_clamped_len(const DecodeParams &p, int b)
     return min(max(__ldg(p.kv_len + b), 0), cap);
 }
 
-template <int NH>
-__global__ void __launch_bounds__(StSmem<NH>::kThreads, 1)
+// Steps (sequence, kv head, chunk) to the next chunk in the order the work is cut in; sequences without
+// tokens are skipped.  Only called while another chunk exists, so a sequence with tokens is always found.
+__device__ __forceinline__ void st_next_chunk(const DecodeParams &p, int B, int &b, int &head, int &chunk, int &len, int &nc)
+{
+    if (++chunk == nc) {
+        chunk = 0;
+        if (++head == p.Hkv) {
+            head = 0;
+            do {
+                ++b;
+                len = (b < B) ? st_clamped_len(p, b) : kStChunk;   // b < B always holds inside a block's range
+                nc = (len + kStChunk - 1) / kStChunk;
+            } while (nc == 0);
+        }
+    }
+}
+
+// Bounded wait until a counter in shared memory (written by another warp of the block) reaches `target`.
+__device__ __noinline__ bool st_wait_count(const volatile int *counter, int target, uint32_t max_tries)
+{
+    while (*counter < target)
+        if (--max_tries == 0u) return false;
+    __threadfence_block();
+    return true;
+}
+
+template <int NH, bool kAppend>
+__global__ void __launch_bounds__(StSmem<NH, kAppend>::kThreads, 1)
 slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __grid_constant__ CUtensorMap map_tail,
                           const DecodeParams p, const int B)
 {
-    using L = StSmem<NH>;
+    using L = StSmem<NH, kAppend>;
     constexpr int N = L::N;
     constexpr int S = L::kStages;
     constexpr int kStGroups = L::kGroups, kStInfoSlots = L::kInfoSlots;
@@ -149,6 +177,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kTmemSlot);
     int *range = reinterpret_cast<int *>(smem + L::kRange);
     volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
+    volatile int *appended = reinterpret_cast<volatile int *>(smem + L::kAppended);
 
     pdl_launch_dependents();   // the merge kernel queued behind this one may be scheduled; it waits for our completion
     if (tid == 0) {
@@ -169,6 +198,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         }
         tc::mbar_init_fence();
         *fail = 0;
+        *appended = 0;
     }
     if (warp == kPW) {
         tc::tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
@@ -215,7 +245,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         };
         const long long i0 = chunks_before(total_tiles * blockIdx.x / gridDim.x);
         const long long i1 = chunks_before(total_tiles * (blockIdx.x + 1) / gridDim.x);
-        int b0 = 0, head0 = 0, chunk0 = 0;
+        int b0 = 0, head0 = 0, chunk0 = 0, nc0 = 1;
         if (i1 > i0) {
             long long prefix = 0;   // chunks of the sequences before `base`
             for (int base = 0; base < B; base += 32) {
@@ -235,6 +265,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     b0 = base + l;
                     head0 = (int)(r / nc_l);
                     chunk0 = (int)(r % nc_l);
+                    nc0 = nc_l;
                     break;
                 }
                 prefix += __shfl_sync(0xffffffffu, incl, 31);
@@ -245,6 +276,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             range[1] = b0;
             range[2] = head0;
             range[3] = chunk0;
+            range[4] = nc0;
         }
     } else if (warp < kPW) {
         // rows of the query operand that belong to no head stay zero for the whole launch
@@ -288,24 +320,23 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             int2 pg = page_ids(b, chunk);
             int stage = 0;
             uint32_t stage_ph = 0;   // parity of the stage's current use
+            // one-call step: list index of the block's first chunk that holds a new token's slot (the last chunk of
+            // the first sequence and head); the consumer warps must have written the block's new rows before it is fetched
+            const int n_first_new = kAppend ? range[4] - 1 - range[3] : -1;
             for (int n = 0; n < cnt; ++n) {
                 const int cb = b, chead = head, cchunk = chunk;
                 const int n_tok = min(kStChunk, len - chunk * kStChunk);
                 const int2 cpg = pg;
                 // ---- the next chunk's coordinates and page ids, requested before this chunk's copies are issued
                 if (n + 1 < cnt) {
-                    if (++chunk == nc) {
-                        chunk = 0;
-                        if (++head == p.Hkv) {
-                            head = 0;
-                            do {
-                                ++b;
-                                len = (b < B) ? st_clamped_len(p, b) : kStChunk;   // b < B always holds inside the range
-                                nc = (len + kStChunk - 1) / kStChunk;
-                            } while (nc == 0);
-                        }
-                    }
+                    st_next_chunk(p, B, b, head, chunk, len, nc);
                     pg = page_ids(min(b, B - 1), chunk);
+                }
+                if (kAppend && n == n_first_new) {
+                    if (!st_wait_count(appended, kPW, ok ? (1u << 20) : 1u)) {
+                        ok = false;
+                        *fail = 1;
+                    }
                 }
                 int page[2] = {cpg.x, cpg.y};
                 int rows16[2];
@@ -450,6 +481,55 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         const int bar_id = 1 + g;
         int q_b = -1, q_head = -1;                                 // whose query rows the operand buffer holds
 
+        if (kAppend) {
+            // ---- one-call step: the block that owns the last chunk of a (sequence, kv head) quantises that pair's
+            //      new K row (lanes 0-15) and V row (lanes 16-31) into slot kv_len - 1 of the cache before its
+            //      producers fetch that chunk; every other chunk of the pair holds older tokens only.  The pairs
+            //      whose last chunk lies in this block's range are dealt to the consumer warps in turn, here, while
+            //      the first tiles are on their way.
+            if (cnt > 0) {
+                pdl_wait();
+                int b = range[1], head = range[2];
+                int len = st_clamped_len(p, b);
+                int nc = range[4];
+                int last = nc - 1 - range[3];   // list index of the pair's last chunk
+                const int kv = lane >> 4, l = lane & 15;
+                for (int r = 0; last < cnt; ++r) {
+                    if (r % kPW == warp) {
+                        const int pos = len - 1;
+                        // a length beyond the page table or the launch's max_kv was clamped: its token has no slot
+                        const bool has_slot = __ldg(p.kv_len + b) == len;
+                        const __nv_bfloat16 *src = (kv ? p.v_new : p.k_new) + ((size_t)b * p.Hkv + head) * kHeadDim;
+                        const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(src) + l);
+                        const int page = __ldg(p.block_table + (size_t)b * p.max_pages_per_seq + (pos >> 7));
+                        float scale;
+                        const uint2 pk = quantize_row16(raw, scale);
+                        if (has_slot && page >= 0 && page < p.num_pages) {
+                            const int slot = pos & (kPageTokens - 1);
+                            int8_t *dst = const_cast<int8_t *>(p.codes) + code_block_offset(page, head, kv, p.Hkv) + (size_t)slot * kHeadDim;
+                            reinterpret_cast<uint2 *>(dst)[l] = pk;
+                            if (l == 0) const_cast<float *>(p.scales)[scale_block_offset(page, head, kv, p.Hkv) + slot] = scale;
+                        }
+                    }
+                    // the next pair with tokens
+                    if (++head == p.Hkv) {
+                        head = 0;
+                        do {
+                            ++b;
+                            len = (b < B) ? st_clamped_len(p, b) : 0;
+                        } while (b < B && len == 0);
+                        if (b >= B) break;
+                        nc = (len + kStChunk - 1) / kStChunk;
+                    }
+                    last += nc;
+                }
+            }
+            // the rows are at device scope and ordered before copies of the async proxy; then the warp is counted
+            __threadfence();
+            tc::fence_proxy_async_global();
+            __syncwarp();
+            if (lane == 0) atomicAdd_block(const_cast<int *>(appended), 1);
+        }
         for (int n = g; n < cnt; n += kStGroups) {
             const int islot = n % kStInfoSlots;
             const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
@@ -639,6 +719,19 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     }
 }
 
+template <int NH, bool kAppend>
+static int launch_stream(dim3 grid, cudaStream_t stream, const CUtensorMap &map_tile, const CUtensorMap &map_tail,
+                         const DecodeParams &p, int B)
+{
+    constexpr int bytes = (int)StSmem<NH, kAppend>::kBytes;
+    const int rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<NH, kAppend>), bytes);
+    if (rc != SLIM_OK) return rc;
+    SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<NH, kAppend>, grid, dim3(StSmem<NH, kAppend>::kThreads), bytes, stream, map_tile,
+                             map_tail, p, B));
+    SLIM_CUDA_TRY(cudaGetLastError());
+    return SLIM_OK;
+}
+
 int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int B, cudaStream_t stream)
 {
     CUtensorMap map_tile, map_tail;
@@ -651,19 +744,14 @@ int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int
     if (rc != SLIM_OK) return rc;
     const long long max_items = (long long)p.n_chunks * p.Hkv * B;
     const unsigned grid = (unsigned)(max_items < sms ? max_items : sms);
+    const dim3 blocks(grid);
+    const bool append = p.k_new != nullptr;
     if (p.G <= 8) {
-        constexpr int bytes = (int)StSmem<8>::kBytes;
-        rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<8>), bytes);
-        if (rc != SLIM_OK) return rc;
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<8>, dim3(grid), dim3(StSmem<8>::kThreads), bytes, stream, map_tile, map_tail, p, B));
-    } else {
-        constexpr int bytes = (int)StSmem<16>::kBytes;
-        rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<16>), bytes);
-        if (rc != SLIM_OK) return rc;
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<16>, dim3(grid), dim3(StSmem<16>::kThreads), bytes, stream, map_tile, map_tail, p, B));
+        if (append) return launch_stream<8, true>(blocks, stream, map_tile, map_tail, p, B);
+        return launch_stream<8, false>(blocks, stream, map_tile, map_tail, p, B);
     }
-    SLIM_CUDA_TRY(cudaGetLastError());
-    return SLIM_OK;
+    if (append) return launch_stream<16, true>(blocks, stream, map_tile, map_tail, p, B);
+    return launch_stream<16, false>(blocks, stream, map_tile, map_tail, p, B);
 }
 
 }  // namespace slim

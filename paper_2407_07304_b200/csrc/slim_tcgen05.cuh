@@ -66,6 +66,9 @@ __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fenc
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
 // Makes generic-proxy writes to shared memory (st.shared, cp.async) visible to the tensor-core (async) proxy.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+// The same for global memory: orders this thread's earlier ordinary stores to global memory before later
+// reads of them by the copy engine (TMA / bulk copies issued after a synchronisation with this thread).
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;\n" ::: "memory"); }
 
 // ---------------------------------------------------------------- tensor memory
 // Allocate / free `cols` (power of two >= 32) TMEM columns; executed by one whole warp.

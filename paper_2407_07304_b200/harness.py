@@ -66,6 +66,19 @@ class LayerRun:
                               self.ws_decode)
         return out
 
+    def decode_step(self, q):
+        """Append the next token of every sequence and attend over the lengthened cache in one library call."""
+        w = self.w
+        k_new = torch.stack([self.k[b][self.pos[b]] for b in range(w.B)]).contiguous()
+        v_new = torch.stack([self.v[b][self.pos[b]] for b in range(w.B)]).contiguous()
+        for b in range(w.B):
+            self.pos[b] += 1
+        q = q.to(self.device).contiguous()
+        out = torch.empty_like(q)
+        slim.slim_decode_step(self.cache, q, k_new, v_new, out, self._i32(self.pos), w.B, max(self.pos), w.Hq,
+                              w.sm_scale, self.ws_decode)
+        return out
+
     # ------------------------------------------------------------------ read-back
     def gather_cache(self, b):
         """Sequence b's cached rows in position order:
@@ -81,9 +94,10 @@ class LayerRun:
         return codes[0], scales[0], codes[1], scales[1]
 
 
-def run_workload(w: Workload, device="cuda", decode_steps=None, block_table=None, num_pages=None):
+def run_workload(w: Workload, device="cuda", decode_steps=None, block_table=None, num_pages=None, one_call_step=False):
     """The workload's full call sequence.  Returns (LayerRun, prefill outputs per sequence or None,
-    {decode step: output [B, Hq, 128]}); decode_steps limits which steps' outputs are kept."""
+    {decode step: output [B, Hq, 128]}); decode_steps limits which steps' outputs are kept.  With one_call_step
+    every decode step is one slim_decode_step call instead of slim_kv_append followed by slim_attn_decode."""
     run = LayerRun(w, device=device, block_table=block_table, num_pages=num_pages)
     out_prefill = None
     if any(n > 0 for n in w.prefill_len):
@@ -93,8 +107,11 @@ def run_workload(w: Workload, device="cuda", decode_steps=None, block_table=None
         run.append(w.bulk_len)
     outs = {}
     for s in range(w.decode_steps):
-        run.append([1] * w.B)
-        o = run.decode(w.q_decode[s])
+        if one_call_step:
+            o = run.decode_step(w.q_decode[s])
+        else:
+            run.append([1] * w.B)
+            o = run.decode(w.q_decode[s])
         if decode_steps is None or s in decode_steps:
             outs[s] = o
     torch.cuda.synchronize()

@@ -60,11 +60,12 @@ def _sample_rows(n, extra, seed):
     return sorted(set(base + more))
 
 
-def _check(w, prefill_rows=None, decode_steps=None):
+def _check(w, prefill_rows=None, decode_steps=None, one_call_step=False):
     """Run the workload on the GPU and compare everything (or the given samples) with the oracle."""
-    from paper_2407_07304_b200 import harness
+    from paper_2407_07304_b200 import binding as slim, harness
     oc = _oracle_cache(w)
-    run, out_prefill, outs = harness.run_workload(w, decode_steps=decode_steps)
+    run, out_prefill, outs = harness.run_workload(w, decode_steps=decode_steps, one_call_step=one_call_step)
+    assert slim.slim_read_status(run.ws_decode) == slim.SLIM_OK
     _assert_cache_bits(run, oc)
     if out_prefill is not None:
         for b in range(w.B):
@@ -86,6 +87,12 @@ def test_workload_small_all_outputs(index, shrink):
     _check(workloads.make_workload(index, shrink=shrink))
 
 
+@pytest.mark.parametrize("index,shrink", [(1, 1), (2, 8), (4, 8), (5, 32)])
+def test_workload_small_one_call_steps(index, shrink):
+    # the decode steps through slim_decode_step: the new token is quantised inside the attention kernel
+    _check(workloads.make_workload(index, shrink=shrink), one_call_step=True)
+
+
 # ---------------------------------------------------------------- full sizes
 def test_c2_full_all_rows():
     _check(workloads.make_workload(2))
@@ -93,6 +100,11 @@ def test_c2_full_all_rows():
 
 def test_c4_full_all_rows():
     _check(workloads.make_workload(4))
+
+
+@pytest.mark.parametrize("index", [2, 4])
+def test_full_one_call_step(index):
+    _check(workloads.make_workload(index), one_call_step=True)
 
 
 def test_c3_full_sampled_rows():
@@ -221,6 +233,33 @@ def test_decode_tail_lengths(Hq, Hkv):
     _check(_custom(B, Hq, Hkv, [0] * B, [n - 1 for n in lens], 1, 700 + Hq))
 
 
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (16, 1), (8, 2)])
+def test_one_call_step_tail_lengths(Hq, Hkv):
+    # the same boundaries with the new token written by the attention kernel itself; at length 1 and 2 the new
+    # token carries most of the softmax weight, so a stale or missing row could not pass
+    lens = [1, 2, 15, 16, 17, 31, 127, 128, 129, 144, 255, 256, 257, 272, 383, 511, 513]
+    B = len(lens)
+    w = _custom(B, Hq, Hkv, [0] * B, [n - 1 for n in lens], 3, 900 + Hq)
+    _check(w, one_call_step=True)
+
+
+def test_one_call_step_equals_append_then_decode_bit_for_bit():
+    from paper_2407_07304_b200 import harness
+    w = workloads.make_workload(4, shrink=8)
+    a, _, outs_a = harness.run_workload(w)
+    b, _, outs_b = harness.run_workload(w, one_call_step=True)
+    for s_ in outs_a:
+        assert torch.equal(outs_a[s_], outs_b[s_])
+    assert torch.equal(a.cache.codes, b.cache.codes) and torch.equal(a.cache.scales, b.cache.scales)
+
+
+def test_one_call_step_many_short_sequences():
+    # more (sequence, kv head) pairs than thread blocks: every block quantises several new rows
+    B = 300
+    lens = [(7 * i) % 40 + 1 for i in range(B)]
+    _check(_custom(B, 4, 2, [0] * B, [n - 1 for n in lens], 2, 950), one_call_step=True)
+
+
 def test_status_words_stay_clear():
     from paper_2407_07304_b200 import binding as slim, harness
     w = workloads.make_workload(1, shrink=2)
@@ -230,7 +269,7 @@ def test_status_words_stay_clear():
 
 
 def test_decode_step_from_host_buffers():
-    # slim_decode_step_host: H2D copies, append, split + merge, D2H copy on one stream
+    # slim_decode_step_host: H2D copies, the one-kernel step, D2H copy on one stream
     from paper_2407_07304_b200 import binding as slim, harness
     w = workloads.make_workload(4, shrink=16)
     run = harness.LayerRun(w)
@@ -243,10 +282,8 @@ def test_decode_step_from_host_buffers():
     q = w.q_decode[0].contiguous().pin_memory()
     out = torch.empty_like(q).pin_memory()
     staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
-    cu_new = torch.arange(B + 1, dtype=torch.int32, device=dev)
-    start = torch.tensor(ctx, dtype=torch.int32, device=dev)
-    kv_len = start + 1
-    slim.slim_decode_step_host(run.cache, q, k_new, v_new, out, staging, cu_new, start, kv_len, B, max(ctx) + 1, Hq,
+    kv_len = torch.tensor(ctx, dtype=torch.int32, device=dev) + 1
+    slim.slim_decode_step_host(run.cache, q, k_new, v_new, out, staging, kv_len, B, max(ctx) + 1, Hq,
                                w.sm_scale, run.ws_decode)
     torch.cuda.synchronize()
     run.pos = [c + 1 for c in ctx]
@@ -255,6 +292,49 @@ def test_decode_step_from_host_buffers():
     for b in range(B):
         want = so.attention(bf16_bits(w.q_decode[0, b:b + 1]), *oc[b], ctx[b] + 1, w.sm_scale)
         _assert_close(out[b:b + 1], want, f"host step seq {b}")
+
+
+def test_decode_step_replayed_from_a_graph():
+    # the host-buffer step recorded by stream capture after one ordinary call; each replay reads the pinned
+    # buffers as they are then, so a replay with the next token's inputs must equal the ordinary call on them
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = workloads.make_workload(1)
+    run = harness.LayerRun(w)
+    run.append([w.total_len(b) - w.decode_steps for b in range(w.B)])
+    dev = run.device
+    B, Hq, Hkv = w.B, w.Hq, w.Hkv
+    ctx = list(run.pos)
+    k_new = torch.stack([w.k[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
+    v_new = torch.stack([w.v[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
+    q = w.q_decode[0].contiguous().pin_memory()
+    out = torch.empty_like(q).pin_memory()
+    staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
+    kv_len = torch.tensor(ctx, dtype=torch.int32, device=dev) + 1
+    side = torch.cuda.Stream()
+
+    def call():
+        slim.slim_decode_step_host(run.cache, q, k_new, v_new, out, staging, kv_len, B, max(ctx) + 1,
+                                   Hq, w.sm_scale, run.ws_decode, side)
+
+    with torch.cuda.stream(side):
+        call()
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+            call()
+        # other inputs for the same cache slot: the replay must pick them up
+        q.copy_(w.q_decode[1])
+        k_new.mul_(-0.5), v_new.mul_(2.0)
+        out.zero_()
+        graph.replay()
+        side.synchronize()
+        replayed = out.clone()
+        out.zero_()
+        call()
+        side.synchronize()
+    assert torch.equal(replayed, out)
+    assert replayed.float().abs().max() > 0
+    assert slim.slim_read_status(run.ws_decode) == 0
 
 
 def test_prefill_scale_jumps_between_key_tiles():
