@@ -276,35 +276,42 @@ def run_ours(args, rank, world, local_rank):
         step_host(i)
     ms_e2e_eager = timed(step_host, args.steps)
     same = torch.equal(out_h, out.cpu())
-    # The same call captured once per cache copy into a CUDA graph (copy in, three kernels, copy out) and replayed:
+    # The same call captured once per cache copy into a CUDA graph (copy in, two kernels, copy out) and replayed:
     # what a serving loop does with a fixed-shape decode step.  The graph reads the pinned buffers at replay time.
-    side = torch.cuda.Stream()
-    graphs = []
-    with torch.cuda.stream(side):
-        for i in range(N_ROT):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
-                slim.slim_decode_step_host(runs[i].cache, q_h, k_h, v_h, out_h, staging, kv_len, B, max_kv, Hq,
-                                           w.sm_scale, ws, side)
-            graphs.append(g)
-        out_h.zero_()
+    def graph_replay_ms():
+        side = torch.cuda.Stream()
+        graphs = []
+        with torch.cuda.stream(side):
+            for i in range(N_ROT):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+                    slim.slim_decode_step_host(runs[i].cache, q_h, k_h, v_h, out_h, staging, kv_len, B, max_kv, Hq,
+                                               w.sm_scale, ws, side)
+                graphs.append(g)
+            out_h.zero_()
 
-        def step_graph(i):
-            graphs[i % N_ROT].replay()
-            side.synchronize()      # the caller needs the result before the next token
+            def step_graph(i):
+                graphs[i % N_ROT].replay()
+                side.synchronize()      # the caller needs the result before the next token
 
-        for i in range(3):
-            step_graph(i)
-        same = same and torch.equal(out_h, out.cpu())
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(side)
-        for i in range(args.steps):
-            step_graph(i)
-        e1.record(side)
-        torch.cuda.synchronize()
-        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
-        barrier()
+            for i in range(3):
+                step_graph(i)
+            ok = torch.equal(out_h, out.cpu())
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for i in range(args.steps):
+                step_graph(i)
+            e1.record(side)
+            torch.cuda.synchronize()
+            ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+            barrier()
+        return ms, ok
+
+    ms_e2e = ms_e2e_eager
+    if not args.no_graph:
+        ms_e2e, same_graph = graph_replay_ms()
+        same = same and same_graph
     clocks = sampler.stop() if sampler else None
 
     # ---- extra single-GPU context numbers (not part of the headline): prefill of workload 3
@@ -341,7 +348,8 @@ def run_ours(args, rank, world, local_rank):
                      "avg_launch_ms": split_avg_ms, "min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
         "e2e": {"value": whole_job_rate(B, args.steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same),
-                "launch": "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step",
+                "launch": ("slim_decode_step_host called and synchronised every step" if args.no_graph else
+                           "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step"),
                 "ms_per_step_without_graph": ms_e2e_eager / args.steps},
         "gpu_launches": 2 * args.steps,
         "clocks": clocks,
@@ -355,9 +363,9 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
-# dram bytes read + written by one slim_decode_stream_kernel launch on this workload, from the ncu capture
-# summarised under profiles/; None while the kernel is newer than the last capture.
-TRAFFIC_PER_LAUNCH = None
+# dram bytes read + written by one slim_decode_stream_kernel launch on this workload (279.91 MB read,
+# 5.26 MB written), from the ncu capture summarised under profiles/.
+TRAFFIC_PER_LAUNCH = 285.17e6
 
 
 def extra_numbers(slim, workloads, dev):
@@ -469,6 +477,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-extra", action="store_true", help="skip the prefill context numbers")
+    ap.add_argument("--no-graph", action="store_true", help="end-to-end leg without CUDA-graph replay (plain calls)")
     ap.add_argument("--extra-only", action="store_true",
                     help="run only the workload-3 prefill/append timings (for profiling that kernel) and print them")
     args = ap.parse_args()
