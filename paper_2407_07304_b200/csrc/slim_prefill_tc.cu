@@ -154,11 +154,51 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     const uint32_t bar0 = sbase + pfl::kMisc + 128;
     auto bar = [&](int which, int idx) { return bar0 + 8u * (uint32_t)(which + idx); };
 
-    if (tid == 0) {
-        for (int i = 0; i < kPfRawStages; ++i) {
-            tc::mbar_init(bar(pfl::RAW_FULL, i), 1);
-            tc::mbar_init(bar(pfl::RAW_EMPTY, i), 128);
+    // The first global-memory round trips of the block start before its set-up is complete: the loader thread
+    // initialises the ring's "full" barriers itself and requests the first raw tiles at once, and the softmax
+    // threads read their query rows into registers; both overlap the barrier set-up and the tensor-memory allocation.
+    int raw_issued = 0;   // loader thread: raw tiles requested so far
+    int page_next = 0;
+    auto request_raw = [&](int i) {
+        const int32_t *bt = p.block_table + (size_t)b * p.max_pages_per_seq;
+        const int slot = i % kPfRawStages, j = i >> 1;
+        const int kv = i & 1;
+        int page = page_next;
+        if (kv == 1 && j + 1 < T) page_next = __ldg(bt + j + 1);   // requested one tile ahead
+        page = (page >= 0 && page < p.num_pages) ? page : 0;
+        const uint32_t dst = sbase + pfl::kRaw + slot * pfl::kRawStage;
+        const uint32_t full = bar(pfl::RAW_FULL, slot);
+        tc::mbar_arrive_expect_tx(full, 16384 + 512);
+        tc::tma_load_2d(dst, &codes_map, 0, ((page * p.Hkv + head) * 2 + kv) * kPageTokens, full);
+        tc::bulk_load(dst + 16384, p.scales + scale_block_offset(page, head, kv, p.Hkv), 512, full);
+        ++raw_issued;
+    };
+    if (warp == 12 && lane == 0) {
+        for (int i = 0; i < kPfRawStages; ++i) tc::mbar_init(bar(pfl::RAW_FULL, i), 1);
+        tc::mbar_init_fence();
+        if (T > 0) {
+            page_next = __ldg(p.block_table + (size_t)b * p.max_pages_per_seq);
+            for (int i = 0; i < min(kPfRawStages, 2 * T); ++i) request_raw(i);   // every stage is free the first time round
         }
+    }
+    uint32_t qw[64];   // softmax threads: this thread's query row (bf16 pairs)
+    if (warp < 8) {
+        const int row = m0 + (warp >> 2) * kPfBM + (tid & 127);
+        if (Tt[warp >> 2] > 0 && row < q_len) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint4 v = __ldg(src + i);
+                qw[4 * i] = v.x, qw[4 * i + 1] = v.y, qw[4 * i + 2] = v.z, qw[4 * i + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 64; ++i) qw[i] = 0u;
+        }
+    }
+
+    if (tid == 0) {
+        for (int i = 0; i < kPfRawStages; ++i) tc::mbar_init(bar(pfl::RAW_EMPTY, i), 128);
         tc::mbar_init(bar(pfl::KF_FULL, 0), 128);
         tc::mbar_init(bar(pfl::KF_EMPTY, 0), 1);
         tc::mbar_init(bar(pfl::VF_FULL, 0), 128);
@@ -185,8 +225,6 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             *fail = 1;
         }
     };
-    int raw_issued = 0;   // loader thread: raw tiles requested so far
-
     // Registers move from the warp groups that need few to the softmax groups, which hold a whole 128-column
     // score row (every warp of a group executes the same setmaxnreg; 2 * 160 + 96 + 96 = 4 * 128 per lane; the split was chosen by measurement).
     if (warp < 8) {
@@ -212,18 +250,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         if (Tmine > 0) {
             // Q row -> fp16 (divided by a power of two near its absmax, so the copy of bf16 is exact),
             // written as the A operand: dims [64 hf, 64 hf + 64) in half hf, 16-byte pieces XOR-swizzled by row
-            uint32_t w[64];
-            if (row_valid) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim);
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const uint4 v = __ldg(src + i);
-                    w[4 * i] = v.x, w[4 * i + 1] = v.y, w[4 * i + 2] = v.z, w[4 * i + 3] = v.w;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 64; ++i) w[i] = 0u;
-            }
+            uint32_t(&w)[64] = qw;   // read before the block's set-up
             float am = 0.f;
 #pragma unroll
             for (int i = 0; i < 64; ++i)
@@ -420,21 +447,9 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     } else if (warp == 12) {
         // =========================================================== loader (one thread)
         if (lane == 0 && T > 0) {
-            const int32_t *bt = p.block_table + (size_t)b * p.max_pages_per_seq;
-            int page_next = __ldg(bt);
-            for (int i = 0; i < 2 * T; ++i) {
-                const int slot = i % kPfRawStages, j = i >> 1;
-                const int kv = i & 1;
-                int page = page_next;
-                if (kv == 1 && j + 1 < T) page_next = __ldg(bt + j + 1);   // requested one tile ahead
-                page = (page >= 0 && page < p.num_pages) ? page : 0;
-                wait(bar(pfl::RAW_EMPTY, slot), ((uint32_t)(i / kPfRawStages) & 1u) ^ 1u);
-                const uint32_t dst = sbase + pfl::kRaw + slot * pfl::kRawStage;
-                const uint32_t full = bar(pfl::RAW_FULL, slot);
-                tc::mbar_arrive_expect_tx(full, 16384 + 512);
-                tc::tma_load_2d(dst, &codes_map, 0, ((page * p.Hkv + head) * 2 + kv) * kPageTokens, full);
-                tc::bulk_load(dst + 16384, p.scales + scale_block_offset(page, head, kv, p.Hkv), 512, full);
-                ++raw_issued;
+            for (int i = kPfRawStages; i < 2 * T; ++i) {   // the first round of the ring was requested during set-up
+                wait(bar(pfl::RAW_EMPTY, i % kPfRawStages), ((uint32_t)(i / kPfRawStages) & 1u) ^ 1u);
+                request_raw(i);
             }
         }
     } else if (warp == 13) {
