@@ -131,16 +131,24 @@ int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out,
  * tokens (the new token's K/V already appended).  Same arithmetic as above with
  * q_len == 1.  The next-token phase is a matrix-vector product bound by memory
  * bandwidth (Section 2.2, Eq. 1); the key range is split across thread blocks
- * and the pieces are merged by the log-sum-exp identity in a second kernel.
+ * and the pieces are merged by the log-sum-exp identity: by the split kernel
+ * itself when its blocks finish where a row has few pieces, otherwise in a
+ * second kernel.
  * A sequence with kv_len[b] == 0 gets zeros.
  *
  *   q, out   device bf16 [B][Hq][128], 16-byte aligned
  *   kv_len   device int32 [B];  max_kv upper bound on kv_len (sizes the launch)
  *   workspace device scratch of at least
  *             slim_workspace_bytes(SLIM_PHASE_DECODE, ...) bytes, 16-byte
- *             aligned; only its first 16 bytes (the status word, see
- *             slim_read_status) need to be zero, the rest need not be initialised
+ *             aligned.  Its first SLIM_WORKSPACE_HEADER_BYTES bytes (the status
+ *             word, see slim_read_status, and the counters of the in-kernel
+ *             merge) must be zero when the workspace is first used (one
+ *             cudaMemset after allocating it); every call leaves the counters
+ *             at zero again, so the same workspace serves any sequence of calls
+ *             on one stream, whatever their shapes.  After a SLIM_ERR_TIMEOUT
+ *             zero the header again.  The rest need not be initialised.
  */
+#define SLIM_WORKSPACE_HEADER_BYTES (16 + 16384 * 4)
 int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out,
                      const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
                      void *workspace, size_t workspace_bytes, void *stream);
@@ -150,12 +158,13 @@ int slim_attn_decode(const slim_cache_t *cache, const void *q, void *out,
  * or time them individually: the split pass (every block: the scores of its key
  * chunk, one softmax over the chunk, the product with V; Section 2.1 order inside
  * the chunk) writes partials into `workspace`; the merge pass combines them into
- * `out`.  Same arguments, validation and workspace as slim_attn_decode;
- * slim_attn_decode(...) == split(..., NULL, NULL, ...) followed by merge(...) on
- * the same stream.  With k_new and v_new (both or neither; as for
+ * `out`.  Same arguments, validation and workspace as slim_attn_decode, whose
+ * result is that of split(..., NULL, NULL, ...) followed by merge(...) on the
+ * same stream (where it merges inside the split kernel, up to the order of the
+ * merge's sums).  With k_new and v_new (both or neither; as for
  * slim_decode_step) the split pass first writes every sequence's new token into
- * slot kv_len[b] - 1: slim_decode_step(...) == split(..., k_new, v_new, ...)
- * followed by merge(...).
+ * slot kv_len[b] - 1: slim_decode_step(...) computes split(..., k_new, v_new,
+ * ...) followed by merge(...).
  */
 int slim_attn_decode_split(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new,
                            const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
@@ -235,8 +244,9 @@ size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
  *    cudaGetSymbolAddress, with that device current); make that first call
  *    before starting any stream capture.
  *  - All calls on a device share the one array, and it keeps whatever the last
- *    call left in it.  Nothing in it has to start at zero: every slot a call
- *    reads was written by that same call's split pass.  Two calls whose kernels
+ *    call left in it.  Its header starts at zero because the array is part of
+ *    the zero-initialised image, and every call leaves it at zero; every other
+ *    slot a call reads was written by that same call's split pass.  Two calls whose kernels
  *    can overlap on the GPU (different streams, no ordering between them) race
  *    on the array and give wrong results; keep calls on one stream or order
  *    them with events.
@@ -253,8 +263,8 @@ int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
  * completion); every such wait gives up after a fixed number of tries, and a kernel whose wait ran out
  * stores SLIM_ERR_TIMEOUT in the first word of its workspace and finishes with undefined output instead of
  * hanging.  slim_read_status synchronises `stream`, reads that word (host <- device) and returns SLIM_OK
- * or SLIM_ERR_TIMEOUT.  The kernels never clear the word: zero the first 16 bytes of a workspace once
- * after allocating it.
+ * or SLIM_ERR_TIMEOUT.  The kernels never clear the word: zero the header of a workspace once after
+ * allocating it (16 bytes for prefill, SLIM_WORKSPACE_HEADER_BYTES for decode).
  */
 int slim_read_status(const void *workspace, void *stream);
 

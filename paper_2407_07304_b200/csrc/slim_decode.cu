@@ -11,6 +11,7 @@
 namespace slim {
 
 constexpr int kChunkTok = 256;   // tokens per partial result (two pages)
+static_assert(kDecodeHeaderBytes == SLIM_WORKSPACE_HEADER_BYTES, "the header size promised in slim.h");
 
 // Second pass: log-sum-exp merge of a row's chunk partials,
 //   M = max m_c;  l = sum l_c 2^(m_c - M);  o = sum O_c 2^(m_c - M) / l.
@@ -90,7 +91,7 @@ size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv)
 {
     (void)Hkv;
     const size_t nc = (size_t)(max_kv + kChunkTok - 1) / kChunkTok;
-    return kDecodeStatusBytes + (size_t)B * Hq * nc * (kHeadDim + 2) * sizeof(float);
+    return kDecodeHeaderBytes + (size_t)B * Hq * nc * (kHeadDim + 2) * sizeof(float);
 }
 
 static DecodeParams make_params(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv,
@@ -112,9 +113,11 @@ static DecodeParams make_params(const slim_cache_t *c, const void *q, const int3
     p.n_chunks = (max_kv + C - 1) / C;
     p.scale_log2e = sm_scale * kLog2e;
     p.status = static_cast<int *>(workspace);
-    p.part_o = reinterpret_cast<float *>(static_cast<char *>(workspace) + kDecodeStatusBytes);
+    p.part_o = reinterpret_cast<float *>(static_cast<char *>(workspace) + kDecodeHeaderBytes);
     p.part_ml = p.part_o + (size_t)B * Hq * p.n_chunks * kHeadDim;
     p.k_new = p.v_new = nullptr;
+    p.out = nullptr;
+    p.counters = nullptr;
     return p;
 }
 
@@ -132,13 +135,26 @@ int launch_decode_split(const slim_cache_t *c, const void *q, const void *k_new,
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
                         const void *workspace, cudaStream_t stream);
 
-// Decode attention: split kernel, then merge kernel.  With k_new / v_new the split kernel first quantises every
-// sequence's new token into slot kv_len - 1 of the cache (the one-call decode step).
+// Decode attention.  With k_new / v_new the split kernel first quantises every sequence's new token into slot
+// kv_len - 1 of the cache (the one-call decode step).  Where a (sequence, kv head) has few partials the split
+// kernel merges them itself when its blocks finish (one warp per pair); otherwise the merge kernel follows.
+constexpr int kInKernelMergeMaxPartials = 32;   // G * chunks of a (sequence, kv head) that one warp merges at the end of a block
+
 int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, void *out,
                   const int32_t *kv_len, int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream)
 {
-    const int rc = launch_decode_split(c, q, k_new, v_new, kv_len, B, max_kv, Hq, sm_scale, workspace, stream);
-    if (rc != SLIM_OK) return rc;
+    int C;
+    DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
+    if (p.n_chunks == 0) return launch_decode_merge(c, out, kv_len, B, max_kv, Hq, workspace, stream);   // rows of zeros
+    p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+    const bool in_kernel = (long long)B * p.Hkv <= kDecodeCounterRows && p.G * p.n_chunks <= kInKernelMergeMaxPartials;
+    if (in_kernel) {
+        p.out = static_cast<__nv_bfloat16 *>(out);
+        p.counters = reinterpret_cast<int *>(static_cast<char *>(workspace) + kDecodeStatusBytes);
+    }
+    const int rc = launch_decode_split_stream(c, p, B, stream);
+    if (rc != SLIM_OK || in_kernel) return rc;
     return launch_decode_merge(c, out, kv_len, B, max_kv, Hq, workspace, stream);
 }
 

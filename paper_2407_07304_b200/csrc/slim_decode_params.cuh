@@ -16,12 +16,21 @@ struct DecodeParams {
     // one-kernel append + split (optional): the new token of every sequence, [B][Hkv][128], quantised into slot
     // kv_len - 1 by the block that owns the sequence's last chunk (null: nothing to append)
     const __nv_bfloat16 *k_new, *v_new;
+    // merge at the end of the split kernel (optional, both or neither): the result [B][Hq][128] and the counters
+    // [B * Hkv] of chunks counted so far per (sequence, kv head); zero before and after every launch
+    __nv_bfloat16 *out;
+    int *counters;
     int Hq, Hkv, G;
     int max_pages_per_seq, num_pages, n_chunks;
     float scale_log2e;        // sm_scale * log2(e)
 };
 
-constexpr size_t kDecodeStatusBytes = 16;   // status word + padding in front of the partials
+// Workspace header in front of the partials: the status word (16 bytes), then the counters of the in-kernel
+// merge.  The header has one size for every shape, so a workspace zeroed once stays valid when the shapes of the
+// calls that use it change.
+constexpr size_t kDecodeStatusBytes = 16;
+constexpr int kDecodeCounterRows = 16384;   // (sequence, kv head) pairs the in-kernel merge can count
+constexpr size_t kDecodeHeaderBytes = kDecodeStatusBytes + (size_t)kDecodeCounterRows * sizeof(int);
 
 int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int B, cudaStream_t stream);
 

@@ -152,7 +152,60 @@ __device__ __noinline__ bool st_wait_count(const volatile int *counter, int targ
     return true;
 }
 
-template <int NH, bool kAppend>
+// Log-sum-exp merge of the nc chunk partials of the G query heads of (sequence b, kv head `head`) by one warp:
+//   M = max m_c;  l = sum l_c 2^(m_c - M);  o = sum O_c 2^(m_c - M) / l   (a lane owns four head dims).
+// The caller has made sure that every partial of the pair is visible; they are read past the L1 cache.
+__device__ __forceinline__ void st_merge_rows(const DecodeParams &p, int b, int head, int nc, int lane)
+{
+    constexpr int kBatch = 12;   // partial outputs requested before the first of them is used
+    for (int h = 0; h < p.G; ++h) {
+        const size_t row = (size_t)b * p.Hq + (size_t)head * p.G + h;
+        const float2 *ml = reinterpret_cast<const float2 *>(p.part_ml) + row * p.n_chunks;
+        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + row * p.n_chunks * kHeadDim) + lane;
+        // every load of the first round is in flight before anything waits for one of them
+        float4 o[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) o[u] = (u < nc) ? __ldcg(po + (size_t)u * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float2 first = (lane < nc) ? __ldcg(ml + lane) : make_float2(-INFINITY, 0.f);
+        float M = first.x;
+        for (int c = lane + 32; c < nc; c += 32) M = fmaxf(M, __ldcg(ml + c).x);
+        M = warp_max(M);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l = 0.f;
+        for (int c0 = 0; c0 < nc; c0 += 32) {
+            float w = 0.f;   // stays 0 for the lanes past the last chunk
+            if (c0 + lane < nc) {
+                const float2 v = (c0 == 0) ? first : __ldcg(ml + c0 + lane);
+                w = exp2f(v.x - M);
+                l = fmaf(v.y, w, l);
+            }
+            for (int j0 = 0; j0 < min(32, nc - c0); j0 += kBatch) {
+                if (c0 + j0 > 0) {
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u)
+                        o[u] = (j0 + u < 32 && c0 + j0 + u < nc) ? __ldcg(po + (size_t)(c0 + j0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const float wj = __shfl_sync(0xffffffffu, w, (j0 + u) & 31);
+                    acc.x = fmaf(o[u].x, wj, acc.x);
+                    acc.y = fmaf(o[u].y, wj, acc.y);
+                    acc.z = fmaf(o[u].z, wj, acc.z);
+                    acc.w = fmaf(o[u].w, wj, acc.w);
+                }
+            }
+        }
+        l = warp_sum(l);
+        const float inv = (l > 0.f) ? 1.f / l : 0.f;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<uint32_t *>(&lo);
+        packed.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(p.out + row * kHeadDim + lane * 4) = packed;
+    }
+}
+
+template <int NH, bool kAppend, bool kMerge>
 __global__ void __launch_bounds__(StSmem<NH, kAppend>::kThreads, 1)
 slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __grid_constant__ CUtensorMap map_tail,
                           const DecodeParams p, const int B)
@@ -704,6 +757,52 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 
     tc::fence_before_sync();
     __syncthreads();
+    if (kMerge) {
+        // ---- the block's partials are written: merge what is complete.  A (sequence, kv head) whose chunks all lie
+        //      in this block's range is merged at once; one that is shared with other blocks is counted in global
+        //      memory (every block adds its number of chunks) and merged by the block whose count completes it.
+        __threadfence();   // this thread's partials are visible device-wide before any count that includes them
+        __syncthreads();
+        if (warp < kPW) {
+            if (cnt > 0) {
+                int b = range[1], head = range[2], first = range[3], nc = range[4];
+                int remaining = cnt;
+                for (int r = 0; remaining > 0; ++r) {
+                    const int mine = min(nc - first, remaining);
+                    if (r % kPW == warp) {
+                        bool complete = mine == nc;
+                        if (!complete) {
+                            int old = 0;
+                            if (lane == 0) old = atomicAdd(p.counters + b * p.Hkv + head, mine);
+                            complete = __shfl_sync(0xffffffffu, old, 0) + mine == nc;
+                            if (complete) {
+                                if (lane == 0) p.counters[b * p.Hkv + head] = 0;   // ready for the next launch
+                                __threadfence();   // the other blocks' counts were seen: their partials are visible after this
+                            }
+                        }
+                        if (complete) st_merge_rows(p, b, head, nc, lane);
+                    }
+                    remaining -= mine;
+                    first = 0;
+                    if (remaining > 0 && ++head == p.Hkv) {
+                        head = 0;
+                        int len;
+                        do {
+                            ++b;
+                            len = (b < B) ? st_clamped_len(p, b) : kStChunk;   // b < B always holds inside the range
+                        } while (len == 0);
+                        nc = (len + kStChunk - 1) / kStChunk;
+                    }
+                }
+            }
+            // sequences without tokens have no chunk and therefore no merge: their rows are zero
+            for (int b = blockIdx.x; b < B; b += gridDim.x) {
+                if (st_clamped_len(p, b) != 0) continue;
+                uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)b * p.Hq * kHeadDim);
+                for (int i = tid; i < p.Hq * (kHeadDim / 8); i += kPW * 32) dst[i] = make_uint4(0, 0, 0, 0);
+            }
+        }
+    }
     if (warp == kPW) {
         if (lane == 0 && *fail != 0) {
             // a wait ran out somewhere: give the copies still in flight a bounded chance to land before the block exits
@@ -719,14 +818,14 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     }
 }
 
-template <int NH, bool kAppend>
+template <int NH, bool kAppend, bool kMerge>
 static int launch_stream(dim3 grid, cudaStream_t stream, const CUtensorMap &map_tile, const CUtensorMap &map_tail,
                          const DecodeParams &p, int B)
 {
     constexpr int bytes = (int)StSmem<NH, kAppend>::kBytes;
-    const int rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<NH, kAppend>), bytes);
+    const int rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_decode_stream_kernel<NH, kAppend, kMerge>), bytes);
     if (rc != SLIM_OK) return rc;
-    SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<NH, kAppend>, grid, dim3(StSmem<NH, kAppend>::kThreads), bytes, stream, map_tile,
+    SLIM_CUDA_TRY(launch_pdl(slim_decode_stream_kernel<NH, kAppend, kMerge>, grid, dim3(StSmem<NH, kAppend>::kThreads), bytes, stream, map_tile,
                              map_tail, p, B));
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
@@ -745,13 +844,21 @@ int launch_decode_split_stream(const slim_cache_t *c, const DecodeParams &p, int
     const long long max_items = (long long)p.n_chunks * p.Hkv * B;
     const unsigned grid = (unsigned)(max_items < sms ? max_items : sms);
     const dim3 blocks(grid);
-    const bool append = p.k_new != nullptr;
+    const bool append = p.k_new != nullptr, merge = p.counters != nullptr;
     if (p.G <= 8) {
-        if (append) return launch_stream<8, true>(blocks, stream, map_tile, map_tail, p, B);
-        return launch_stream<8, false>(blocks, stream, map_tile, map_tail, p, B);
+        if (merge) {
+            if (append) return launch_stream<8, true, true>(blocks, stream, map_tile, map_tail, p, B);
+            return launch_stream<8, false, true>(blocks, stream, map_tile, map_tail, p, B);
+        }
+        if (append) return launch_stream<8, true, false>(blocks, stream, map_tile, map_tail, p, B);
+        return launch_stream<8, false, false>(blocks, stream, map_tile, map_tail, p, B);
     }
-    if (append) return launch_stream<16, true>(blocks, stream, map_tile, map_tail, p, B);
-    return launch_stream<16, false>(blocks, stream, map_tile, map_tail, p, B);
+    if (merge) {
+        if (append) return launch_stream<16, true, true>(blocks, stream, map_tile, map_tail, p, B);
+        return launch_stream<16, false, true>(blocks, stream, map_tile, map_tail, p, B);
+    }
+    if (append) return launch_stream<16, true, false>(blocks, stream, map_tile, map_tail, p, B);
+    return launch_stream<16, false, false>(blocks, stream, map_tile, map_tail, p, B);
 }
 
 }  // namespace slim
