@@ -223,8 +223,8 @@ def run_ours(args, rank, world, local_rank):
     stream = torch.cuda.current_stream()
 
     def step(i):
-        # one call, two kernels: the split kernel quantises the new token's K/V rows into the cache before it reads
-        # them, the merge kernel combines the partial results
+        # one call, one kernel: it quantises the new token's K/V rows into the cache before it reads them, streams
+        # the cache once and merges its own partial results as its blocks finish
         slim.slim_decode_step(runs[i % N_ROT].cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
 
     def timed(fn, steps):
@@ -247,15 +247,14 @@ def run_ours(args, rank, world, local_rank):
         time.sleep(0.1)
     # ---- headline: device-resident inputs, whole step
     ms_total = timed(step, args.steps)
-    # ---- per-kernel: the step's split kernel (new rows written, cache streamed) alone, events around every launch
+    # ---- per-kernel: events around every launch of the step's kernel (back to back in the loop above a launch's
+    #      set-up overlaps the end of the one before it; here it does not)
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     barrier()
     for i in range(args.steps):
-        c = runs[i % N_ROT].cache
         evs[i][0].record(stream)
-        slim.slim_attn_decode_split(c, q, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream, k_new=k_new, v_new=v_new)
+        step(i)
         evs[i][1].record(stream)
-        slim.slim_attn_decode_merge(c, out, kv_len, B, max_kv, Hq, ws, stream)
     torch.cuda.synchronize()
     split_ms = [a.elapsed_time(b) for a, b in evs]
     # ---- end to end: host (pinned) inputs and outputs through slim_decode_step_host
@@ -276,7 +275,7 @@ def run_ours(args, rank, world, local_rank):
         step_host(i)
     ms_e2e_eager = timed(step_host, args.steps)
     same = torch.equal(out_h, out.cpu())
-    # The same call captured once per cache copy into a CUDA graph (copy in, two kernels, copy out) and replayed:
+    # The same call captured once per cache copy into a CUDA graph (copy in, one kernel, copy out) and replayed:
     # what a serving loop does with a fixed-shape decode step.  The graph reads the pinned buffers at replay time.
     def graph_replay_ms():
         side = torch.cuda.Stream()
@@ -326,8 +325,12 @@ def run_ours(args, rank, world, local_rank):
     cache_bytes = sum(kv_len_host) * Hkv * ROW_BYTES
     # whole step: cache read once, Q in, O out, new K/V rows read as bf16 and written as codes + scales
     step_bytes = cache_bytes + 2 * B * Hq * 256 + B * Hkv * (2 * 256 + ROW_BYTES)
-    split_bytes = step_bytes - B * Hq * 256      # the split kernel: all of that but the final output
-    split_avg_ms = statistics.mean(split_ms)
+    split_bytes = step_bytes                     # the step is one kernel
+    # The step is one kernel, so its average launch duration over the timed region is the step time: K launches
+    # between two events on the launching stream.  Launched back to back a kernel's set-up overlaps the end of the
+    # launch before it (programmatic dependent launch); with an event pair around every single launch it does
+    # not, which is the `isolated_launch_ms` figure.
+    split_avg_ms = ms_total / args.steps
     achieved = split_bytes / (split_avg_ms * 1e-3) / 1e9
     h2d = (B * Hq + 2 * B * Hkv) * 128 * 2
     d2h = B * Hq * 128 * 2
@@ -345,13 +348,14 @@ def run_ours(args, rank, world, local_rank):
         "roofline": {"bound": "hbm", "kernel": "slim_decode_stream_kernel", "achieved": achieved, "peak": hbm_peak,
                      "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_8tbs": achieved / 8000.0, "bytes_per_launch": split_bytes,
-                     "avg_launch_ms": split_avg_ms, "min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
+                     "avg_launch_ms": split_avg_ms, "isolated_launch_ms": statistics.mean(split_ms),
+                     "isolated_min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
         "e2e": {"value": whole_job_rate(B, args.steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same),
                 "launch": ("slim_decode_step_host called and synchronised every step" if args.no_graph else
                            "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step"),
                 "ms_per_step_without_graph": ms_e2e_eager / args.steps},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": args.steps,
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu:
@@ -363,9 +367,9 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
-# dram bytes read + written by one slim_decode_stream_kernel launch on this workload (279.91 MB read,
-# 5.26 MB written), from the ncu capture summarised under profiles/.
-TRAFFIC_PER_LAUNCH = 285.17e6
+# dram bytes read + written by one slim_decode_stream_kernel launch on this workload (281.29 MB read,
+# 5.82 MB written), from the ncu capture summarised under profiles/.
+TRAFFIC_PER_LAUNCH = 287.11e6
 
 
 def extra_numbers(slim, workloads, dev):
