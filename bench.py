@@ -353,7 +353,8 @@ def run_ours(args, rank, world, local_rank):
         "e2e": {"value": whole_job_rate(B, args.steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same),
                 "launch": ("slim_decode_step_host called and synchronised every step" if args.no_graph else
-                           "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step"),
+                           "slim_decode_step_host captured in a CUDA graph per cache copy, replayed and synchronised every step")
+                          + "; inputs: one host-to-device copy, result: written by the kernel into the pinned host buffer",
                 "ms_per_step_without_graph": ms_e2e_eager / args.steps},
         "gpu_launches": args.steps,
         "clocks": clocks,

@@ -201,7 +201,9 @@ int slim_decode_step(const slim_cache_t *cache, const void *q, const void *k_new
  * valid and out_host must not be read until the stream has been synchronised.
  *
  * If q_host, k_new_host and v_new_host lie back to back in one allocation (in that order) they are copied with
- * one transfer instead of three.
+ * one transfer instead of three.  If out_host is pinned memory that the device can address (cudaHostAlloc,
+ * cudaHostRegister) and 16-byte aligned, the kernel writes the result straight into it and no copy back is
+ * issued; otherwise the result goes through `staging` and a device -> host copy.
  *
  * The call synchronises nothing and allocates nothing.  After one ordinary call with the same cache and shapes
  * (which creates the tensor map and sets the kernels' attributes) it may be recorded by stream capture into a

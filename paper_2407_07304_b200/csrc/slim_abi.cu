@@ -172,9 +172,19 @@ SLIM_EXPORT int slim_decode_step_host(const slim_cache_t *cache, const void *q_h
         SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, hk, kv_bytes, cudaMemcpyHostToDevice, st));
         SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, hv, kv_bytes, cudaMemcpyHostToDevice, st));
     }
-    rc = launch_decode(cache, d_q, d_k, d_v, d_o, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
+    // A pinned host buffer is mapped into the device's address space: the kernel then writes the result straight
+    // into it (visible to the host once the stream has been synchronised) and the copy back is not needed.
+    void *d_out = d_o;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+        attr.devicePointer != nullptr && ((uintptr_t)attr.devicePointer & 15) == 0) {
+        d_out = attr.devicePointer;
+    } else {
+        (void)cudaGetLastError();   // an unregistered host pointer is not an error here: it takes the copy
+    }
+    rc = launch_decode(cache, d_q, d_k, d_v, d_out, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
     if (rc != SLIM_OK) return rc;
-    SLIM_CUDA_TRY(cudaMemcpyAsync(out_host, d_o, q_bytes, cudaMemcpyDeviceToHost, st));
+    if (d_out == d_o) SLIM_CUDA_TRY(cudaMemcpyAsync(out_host, d_o, q_bytes, cudaMemcpyDeviceToHost, st));
     return SLIM_OK;
 }
 
