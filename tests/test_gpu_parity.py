@@ -268,8 +268,10 @@ def test_status_words_stay_clear():
     assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
 
 
-def test_decode_step_from_host_buffers():
-    # slim_decode_step_host: H2D copies, the one-kernel step, D2H copy on one stream
+@pytest.mark.parametrize("pinned_out", [True, False])
+def test_decode_step_from_host_buffers(pinned_out):
+    # slim_decode_step_host: H2D copy, the one-kernel step, and the result either written by the kernel into the
+    # pinned host buffer or, for ordinary host memory, copied back through the staging buffer
     from paper_2407_07304_b200 import binding as slim, harness
     w = workloads.make_workload(4, shrink=16)
     run = harness.LayerRun(w)
@@ -280,7 +282,7 @@ def test_decode_step_from_host_buffers():
     k_new = torch.stack([w.k[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
     v_new = torch.stack([w.v[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
     q = w.q_decode[0].contiguous().pin_memory()
-    out = torch.empty_like(q).pin_memory()
+    out = torch.zeros_like(q).pin_memory() if pinned_out else torch.zeros(q.shape, dtype=q.dtype)
     staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
     kv_len = torch.tensor(ctx, dtype=torch.int32, device=dev) + 1
     slim.slim_decode_step_host(run.cache, q, k_new, v_new, out, staging, kv_len, B, max(ctx) + 1, Hq,
