@@ -187,6 +187,7 @@ def slim_attn_decode_merge(cache, out, kv_len, B, max_kv, Hq, workspace, stream=
 
 
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
+WORKSPACE_HEADER_BYTES = 16 + 16384 * 4   # zero at first use (SLIM_WORKSPACE_HEADER_BYTES)
 
 
 def slim_attn_decode_static(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, stream=None):

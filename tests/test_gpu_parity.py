@@ -253,6 +253,31 @@ def test_one_call_step_equals_append_then_decode_bit_for_bit():
     assert torch.equal(a.cache.codes, b.cache.codes) and torch.equal(a.cache.scales, b.cache.scales)
 
 
+def test_one_workspace_serves_calls_of_different_shapes():
+    # the decode workspace's header (status word + the in-kernel merge's counters) is zeroed once; every call
+    # leaves it at zero, so calls of other shapes can follow in the same workspace without zeroing it again
+    from paper_2407_07304_b200 import binding as slim, harness
+    shapes = [_custom(5, 4, 4, [0] * 5, [300, 511, 40, 700, 256], 2, 960),       # in-kernel merge, pairs shared between blocks
+              _custom(2, 16, 1, [0] * 2, [9000, 100], 1, 961),                    # too many partials per pair: merge kernel
+              _custom(40, 2, 2, [0] * 40, [(13 * i) % 90 + 1 for i in range(40)], 2, 962)]
+    big = max(slim.slim_workspace_bytes(slim.PHASE_DECODE, w.B, w.Hq, w.Hkv, 1, max(w.total_len(b) for b in range(w.B)))
+              for w in shapes)
+    ws = torch.zeros(big, dtype=torch.uint8, device="cuda")
+    for rounds in range(2):
+        for w in shapes:
+            run = harness.LayerRun(w)
+            run.ws_decode = ws
+            run.append(w.bulk_len)
+            oc = _oracle_cache(w)
+            for s_ in range(w.decode_steps):
+                o = run.decode_step(w.q_decode[s_])
+                for b in range(w.B):
+                    want = so.attention(bf16_bits(w.q_decode[s_, b:b + 1]), *oc[b], w.bulk_len[b] + s_ + 1, w.sm_scale)
+                    _assert_close(o[b:b + 1], want, f"{w.name} step {s_} seq {b}")
+            torch.cuda.synchronize()
+            assert not ws[:slim.WORKSPACE_HEADER_BYTES].any(), "the header is not back at zero"
+
+
 def test_one_call_step_many_short_sequences():
     # more (sequence, kv head) pairs than thread blocks: every block quantises several new rows
     B = 300
