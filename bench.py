@@ -439,8 +439,8 @@ def extra_numbers(slim, workloads, dev):
         return {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
                 "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "cache": label}
 
-    def prefill_numbers(index):
-        w = workloads.make_workload(index)
+    def prefill_numbers(index, shrink=1, reps=3):
+        w = workloads.make_workload(index, shrink=shrink)
         r = LayerRun(w, device=dev)
         n = w.prefill_len[0]
         r.append(w.prefill_len)
@@ -452,10 +452,28 @@ def extra_numbers(slim, workloads, dev):
         def pf():
             slim.slim_attn_prefill(r.cache, q5, o5, cu5, kv5, 1, n, n, w.Hq, w.sm_scale, r.ws_prefill, stream)
 
-        ms = time_it(pf, 3)
+        ms = time_it(pf, reps)
         fl = 4 * 128 * w.Hq * n * (n + 1) // 2
-        return {"workload": w.name, "ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
+        return {"workload": w.name, "tokens": n, "ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
                 "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
+
+    def step_numbers(index, label):
+        """slim_decode_step (append of one token per sequence + decode in one call) at the workload's final context."""
+        w = workloads.make_workload(index)
+        r = LayerRun(w, device=dev)
+        ctx = [w.total_len(b) - 1 for b in range(w.B)]
+        r.append(ctx)
+        kn = torch.stack([r.k[b][ctx[b]] for b in range(w.B)]).contiguous()
+        vn = torch.stack([r.v[b][ctx[b]] for b in range(w.B)]).contiguous()
+        qd = w.q_decode[0].to(dev).contiguous()
+        od = torch.empty_like(qd)
+        kvl = torch.tensor([c + 1 for c in ctx], dtype=torch.int32, device=dev)
+
+        def st():
+            slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, stream)
+
+        ms = time_it(st, 50)
+        return {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "cache": label}
 
     more = {}
     if not os.environ.get("SLIM_BENCH_SHORT"):
@@ -463,7 +481,11 @@ def extra_numbers(slim, workloads, dev):
                 "decode_c5": decode_numbers(5, 1, "17 MB, L2-resident: a latency number, not an HBM number"),
                 "decode_c1": decode_numbers(1, 1, "2 MB, L2-resident: a latency number, not an HBM number"),
                 "prefill_c5": prefill_numbers(5),
-                "prefill_c1": prefill_numbers(1)}
+                "prefill_c1": prefill_numbers(1),
+                "step_c1": step_numbers(1, "2 MB, L2-resident: a latency number"),
+                "step_c5": step_numbers(5, "17 MB, L2-resident: a latency number"),
+                # one sequence, 32 heads, the sequence lengths of the paper's Table 3 (256 ... 4096 tokens)
+                "prefill_sweep": [prefill_numbers(3, shrink=k, reps=10) for k in (32, 16, 8, 4, 2)]}
     return {**more, **{
         "prefill_c3": {"workload": w3.name, "ms": ms_prefill, "tflops": flops / (ms_prefill * 1e-3) / 1e12,
                        "frac_of_bf16_peak": flops / (ms_prefill * 1e-3) / 1e12 / bf16_peak,
