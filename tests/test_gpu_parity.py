@@ -107,6 +107,12 @@ def test_full_one_call_step(index):
     _check(workloads.make_workload(index), one_call_step=True)
 
 
+def test_c5_full_one_call_steps_sampled():
+    # 32 705 ... 32 768 cached tokens, 16 query heads per kv head: more partials per pair than the split kernel merges
+    # itself, so the one-call step here is the split kernel (new rows written inside) followed by the merge kernel
+    _check(workloads.make_workload(5), prefill_rows=8, decode_steps={0, 63}, one_call_step=True)
+
+
 def test_c3_full_sampled_rows():
     _check(workloads.make_workload(3), prefill_rows=48)
 
