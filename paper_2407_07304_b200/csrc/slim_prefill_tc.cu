@@ -48,7 +48,8 @@ constexpr uint32_t kVf = kKf + 32768;           // fp16 V tile: two 64-dim halve
 constexpr uint32_t kRaw = kVf + 32768;          // raw stages: 16 KB INT8 tile + 512 B scales (+ pad)
 constexpr uint32_t kRawStage = 17408;
 constexpr uint32_t kMisc = kRaw + kPfRawStages * kRawStage;
-constexpr uint32_t kBytes = kMisc + 512;
+constexpr uint32_t kRowScale = kMisc + 512;     // float[2][128]: row scale of every query row (written by the thread that converts the row)
+constexpr uint32_t kBytes = kRowScale + 1024;
 // kMisc: floats by parity of the key tile j: [0,2) kexp, [2,4) log2 vexp, [12,14) 1 / vexp; converter warp maxima
 //        [4,12) for K tiles and [20,28) for V tiles; byte 64: tensor-memory address; byte 72: failure flag;
 //        byte 128..: mbarriers
@@ -181,19 +182,21 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             for (int i = 0; i < min(kPfRawStages, 2 * T); ++i) request_raw(i);   // every stage is free the first time round
         }
     }
-    uint32_t qw[64];   // softmax threads: this thread's query row (bf16 pairs)
+    // Query rows are read coalesced: sixteen lanes read one row's 256 bytes, so a warp's load covers two whole rows
+    // (a thread per row would touch 32 rows with 16 bytes each, and the load/store unit would be busy with those
+    // scattered sectors for microseconds while the set-up's own shared-memory traffic queues behind them).  A warp
+    // of query tile t converts the tile's rows 32 (warp & 3) + 2 i + (lane >> 4), i = 0..15; a lane holds piece
+    // lane & 15 (eight dims) of each.
+    uint4 qv[16];
     if (warp < 8) {
-        const int row = m0 + (warp >> 2) * kPfBM + (tid & 127);
-        if (Tt[warp >> 2] > 0 && row < q_len) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim);
+        const int t = warp >> 2;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const uint4 v = __ldg(src + i);
-                qw[4 * i] = v.x, qw[4 * i + 1] = v.y, qw[4 * i + 2] = v.z, qw[4 * i + 3] = v.w;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 64; ++i) qw[i] = 0u;
+        for (int i = 0; i < 16; ++i) {
+            const int rr = (warp & 3) * 32 + 2 * i + (lane >> 4);
+            const int row = m0 + t * kPfBM + rr;
+            qv[i] = make_uint4(0, 0, 0, 0);
+            if (Tt[t] > 0 && row < q_len)
+                qv[i] = __ldg(reinterpret_cast<const uint4 *>(p.q + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim) + (lane & 15));
         }
     }
 
@@ -214,6 +217,36 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         *fail = 0;
     }
     if (warp == 13) tc::tmem_alloc(smem_u32(tmem_slot), kPfTmemCols);
+    if (warp < 8 && Tt[warp >> 2] > 0) {
+        // (needs nothing of the set-up: it overlaps the barrier initialisation and the tensor-memory allocation)
+        const int t = warp >> 2;
+        // Q rows -> fp16 (a row is divided by a power of two near its absmax, so the copy of bf16 is exact),
+        // written as the A operand: dims [64 hf, 64 hf + 64) in half hf, 16-byte pieces XOR-swizzled by row
+        float *row_scale = reinterpret_cast<float *>(smem + pfl::kRowScale) + t * kPfBM;
+        const int piece = lane & 15;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int rr = (warp & 3) * 32 + 2 * i + (lane >> 4);
+            const uint32_t w[4] = {qv[i].x, qv[i].y, qv[i].z, qv[i].w};
+            float am = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                am = fmaxf(am, fmaxf(fabsf(bf16_bits_to_float(w[k] & 0xFFFFu)), fabsf(bf16_bits_to_float(w[k] >> 16))));
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));   // the row's sixteen lanes
+            const float p2 = pow2_floor(am);
+            const float inv = pow2_recip(p2);
+            uint32_t hw[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                hw[k] = pack_half2(bf16_bits_to_float(w[k] & 0xFFFFu) * inv, bf16_bits_to_float(w[k] >> 16) * inv);
+            const uint32_t off = pfl::kQ + (uint32_t)t * 32768u + (uint32_t)(piece >> 3) * 16384u + (uint32_t)rr * 128u +
+                                 (uint32_t)(((piece & 7) ^ (rr & 7)) << 4);
+            *reinterpret_cast<uint4 *>(smem + off) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+            if (piece == 0) row_scale[rr] = p2 * p.scale_log2e;
+        }
+        tc::fence_proxy_async();
+    }
     tc::fence_before_sync();
     __syncthreads();
     tc::fence_after_sync();
@@ -248,27 +281,9 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         const uint32_t tO = tmem + lane_base + kPfTmemO + (uint32_t)t * 128u;
         float rs = 0.f;
         if (Tmine > 0) {
-            // Q row -> fp16 (divided by a power of two near its absmax, so the copy of bf16 is exact),
-            // written as the A operand: dims [64 hf, 64 hf + 64) in half hf, 16-byte pieces XOR-swizzled by row
-            uint32_t(&w)[64] = qw;   // read before the block's set-up
-            float am = 0.f;
-#pragma unroll
-            for (int i = 0; i < 64; ++i)
-                am = fmaxf(am, fmaxf(fabsf(bf16_bits_to_float(w[i] & 0xFFFFu)), fabsf(bf16_bits_to_float(w[i] >> 16))));
-            const float p2 = pow2_floor(am);
-            const float inv = pow2_recip(p2);
-            rs = p2 * p.scale_log2e;
-#pragma unroll
-            for (int i = 0; i < 64; ++i)
-                w[i] = pack_half2(bf16_bits_to_float(w[i] & 0xFFFFu) * inv, bf16_bits_to_float(w[i] >> 16) * inv);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const uint32_t off = pfl::kQ + (uint32_t)t * 32768u + (uint32_t)(i >> 3) * 16384u + (uint32_t)r * 128u +
-                                     (uint32_t)(((i & 7) ^ (r & 7)) << 4);
-                *reinterpret_cast<uint4 *>(smem + off) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-            }
-            tc::fence_proxy_async();
+            // the tile's rows were converted before the set-up's barrier, which also ordered the row scales
             tc::mbar_arrive(bar(pfl::Q_FULL, t));
+            rs = reinterpret_cast<const float *>(smem + pfl::kRowScale)[t * kPfBM + r];
         }
 
         float m_run = -INFINITY, l_run = 0.f;
