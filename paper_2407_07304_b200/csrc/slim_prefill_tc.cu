@@ -379,25 +379,37 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             __syncwarp();
             tc::fence_after_sync();
             const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
-            uint4 *dst = reinterpret_cast<uint4 *>(p.out + ((size_t)(q0 + row) * p.Hq + h) * kHeadDim);
+            // The rows go out coalesced: every thread puts its bf16 row into the tile's Q buffer (no score MMA of this
+            // block reads it any more), 16-byte piece i of row r rotated to piece slot (i + r) mod 16 so that neither
+            // these stores nor the loads below collide on banks; then sixteen lanes write one row's 256 bytes, two rows
+            // per warp store.  A warp reads back only rows its own threads wrote.
+            unsigned char *stage = smem + pfl::kQ + (uint32_t)t * 32768u;
 #pragma unroll
             for (int c4 = 0; c4 < 4; ++c4) {
                 uint32_t v[32];
                 tc::tmem_ld32(tO + c4 * 32, v);
                 tc::tmem_ld_wait();
-                if (row_valid) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint32_t o4[4];
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t o4[4];
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            __nv_bfloat162 x = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * k]) * inv_l,
-                                                                     __uint_as_float(v[8 * i + 2 * k + 1]) * inv_l);
-                            o4[k] = *reinterpret_cast<uint32_t *>(&x);
-                        }
-                        dst[c4 * 4 + i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                    for (int k = 0; k < 4; ++k) {
+                        __nv_bfloat162 x = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * k]) * inv_l,
+                                                                 __uint_as_float(v[8 * i + 2 * k + 1]) * inv_l);
+                        o4[k] = *reinterpret_cast<uint32_t *>(&x);
                     }
+                    *reinterpret_cast<uint4 *>(stage + r * 256 + (((c4 * 4 + i + r) & 15) << 4)) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
                 }
+            }
+            __syncwarp();
+            const int piece = lane & 15;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int rr = (warp & 3) * 32 + 2 * i + (lane >> 4);
+                const int orow = m0 + t * kPfBM + rr;
+                const uint4 o = *reinterpret_cast<const uint4 *>(stage + rr * 256 + (((piece + rr) & 15) << 4));
+                if (orow < q_len)
+                    reinterpret_cast<uint4 *>(p.out + ((size_t)(q0 + orow) * p.Hq + h) * kHeadDim)[piece] = o;
             }
         } else if (row_valid) {
             // a row that sees no key
