@@ -3,66 +3,94 @@
 // The kernel is bound by memory traffic (256 bytes read, 132 written per row), so it is laid out to
 // keep many 16-byte loads in flight per thread and to spend few instructions per element:
 //
-//  * 16 lanes own one row (a lane holds eight consecutive dims: one 16-byte load, one 8-byte store of
-//    codes); a block of 256 threads handles 64 consecutive rows, four per half-warp, all loads issued
-//    before any arithmetic.
+//  * 16 / NV lanes own one row (a lane holds NV pieces of eight consecutive dims: a 16-byte load and an
+//    8-byte store of codes each); a block of 256 threads handles 64 * NV consecutive rows, four per group
+//    of lanes, all loads issued before any arithmetic.
 //  * the row quantiser itself (exact round-half-even codes, bit for bit reproducible) is in slim_quant.cuh.
 #include "slim_common.cuh"
 #include "slim_quant.cuh"
 
 namespace slim {
 
-constexpr int kAppendThreads = 256;
-constexpr int kAppendRowsPerGroup = 4;                                       // rows in flight per half-warp
-constexpr int kAppendRowsPerBlock = (kAppendThreads / 16) * kAppendRowsPerGroup;   // 64
+#ifndef SLIM_APPEND_NV
+#define SLIM_APPEND_NV 4   // four lanes per row: the per-row work (shuffles, reciprocal, addresses) is shared by 32 values per lane
+#endif
+#ifndef SLIM_APPEND_ROWS
+#define SLIM_APPEND_ROWS 1
+#endif
+#ifndef SLIM_APPEND_THREADS
+#define SLIM_APPEND_THREADS 256
+#endif
+#ifdef SLIM_APPEND_MINBLOCKS
+#define SLIM_APPEND_BOUNDS __launch_bounds__(SLIM_APPEND_THREADS, SLIM_APPEND_MINBLOCKS)
+#else
+#define SLIM_APPEND_BOUNDS __launch_bounds__(SLIM_APPEND_THREADS)
+#endif
+constexpr int kAppendThreads = SLIM_APPEND_THREADS;
+constexpr int kAppendRowsPerGroup = SLIM_APPEND_ROWS;   // rows in flight per group of lanes
 
-// grid = (ceil(max_new * Hkv / 64), B, 2 [K, V]); row index = token * Hkv + head within the sequence's new rows.
-__global__ void __launch_bounds__(kAppendThreads)
+// NV = 16-byte loads per lane and row: 16 / NV lanes own a row.
+// grid = (ceil(max_new * Hkv / rows per block), B, 2 [K, V]); row index = token * Hkv + head within the
+// sequence's new rows.  step_tok / step_head = quotient and remainder of the block's group count by Hkv.
+template <int NV>
+__global__ void SLIM_APPEND_BOUNDS
 slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
                    const int32_t *__restrict__ block_table,
                    const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
                    const int32_t *__restrict__ cu_new, const int32_t *__restrict__ start_pos,
-                   int Hkv, int max_pages_per_seq, int num_pages)
+                   int Hkv, int max_pages_per_seq, int num_pages, int step_tok, int step_head)
 {
+    constexpr int kLanes = 16 / NV;                       // lanes per row
+    constexpr int kGroups = kAppendThreads / kLanes;      // rows the block handles per step
+    constexpr int kRowsPerBlock = kGroups * kAppendRowsPerGroup;
     pdl_launch_dependents();   // a decode kernel queued behind this one may run its set-up meanwhile
     const int b = blockIdx.y;
     const int kv = blockIdx.z;
-    const int hw = threadIdx.x >> 4, l = threadIdx.x & 15;
+    const int g = threadIdx.x / kLanes, l = threadIdx.x % kLanes;
     const int row0 = __ldg(cu_new + b);
     // 32-bit row arithmetic (the host checks that max_new * Hkv fits): 64-bit divisions would cost more
     // instructions than the quantiser itself
     const int n_rows = (__ldg(cu_new + b + 1) - row0) * Hkv;
-    const int first = (int)blockIdx.x * kAppendRowsPerBlock;
+    const int first = (int)blockIdx.x * kRowsPerBlock;
     if (first >= n_rows) return;
     const int start = __ldg(start_pos + b);
     const uint4 *src = reinterpret_cast<const uint4 *>((kv ? v_new : k_new) + (size_t)row0 * Hkv * kHeadDim);
 
-    // ---- every load first: the rows' data and the page ids of their destinations
-    uint4 raw[kAppendRowsPerGroup];
+    // ---- every load first: the rows' data and the page ids of their destinations.  One division per thread:
+    // the rows of a thread are kGroups apart, so token and head advance by fixed steps.
+    uint4 raw[kAppendRowsPerGroup][NV];
     int page[kAppendRowsPerGroup], head[kAppendRowsPerGroup], slot[kAppendRowsPerGroup];
+    int tok = (int)((unsigned)(first + g) / (unsigned)Hkv);
+    int hd = first + g - tok * Hkv;
 #pragma unroll
     for (int i = 0; i < kAppendRowsPerGroup; ++i) {
-        const int r = first + i * 16 + hw;     // the block's half-warps cover 16 consecutive rows per step
+        const int r = first + i * kGroups + g;     // the block's groups cover kGroups consecutive rows per step
         page[i] = -1;
-        raw[i] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) raw[i][v] = make_uint4(0, 0, 0, 0);
         if (r < n_rows) {
-            raw[i] = __ldg(src + (size_t)r * 16 + l);
-            const int tok = (int)((unsigned)r / (unsigned)Hkv);
-            head[i] = r - tok * Hkv;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) raw[i][v] = __ldg(src + (size_t)r * 16 + v * kLanes + l);
+            head[i] = hd;
             const int pos = start + tok;
             slot[i] = pos & (kPageTokens - 1);
             const int page_idx = pos >> 7;
             if (pos >= 0 && page_idx < max_pages_per_seq) page[i] = __ldg(block_table + (size_t)b * max_pages_per_seq + page_idx);
         }
+        tok += step_tok;
+        hd += step_head;
+        if (hd >= Hkv) { hd -= Hkv; ++tok; }
     }
 
 #pragma unroll
     for (int i = 0; i < kAppendRowsPerGroup; ++i) {
         float scale;
-        const uint2 pk = quantize_row16(raw[i], scale);
+        uint2 pk[NV];
+        quantize_row<NV>(raw[i], pk, scale);
         if (page[i] >= 0 && page[i] < num_pages) {
             int8_t *dst = codes + code_block_offset(page[i], head[i], kv, Hkv) + (size_t)slot[i] * kHeadDim;
-            reinterpret_cast<uint2 *>(dst)[l] = pk;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) reinterpret_cast<uint2 *>(dst)[v * kLanes + l] = pk[v];
             if (l == 0) scales[scale_block_offset(page[i], head[i], kv, Hkv) + slot[i]] = scale;
         }
     }
@@ -71,14 +99,16 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
 int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
                   const int32_t *start_pos, int B, int max_new, cudaStream_t stream)
 {
+    constexpr int NV = SLIM_APPEND_NV;
+    constexpr int kGroups = kAppendThreads / (16 / NV), kRowsPerBlock = kGroups * kAppendRowsPerGroup;
     const long long rows = (long long)max_new * c->num_kv_heads;
-    const long long blocks = (rows + kAppendRowsPerBlock - 1) / kAppendRowsPerBlock;
+    const long long blocks = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
     if (rows > 0x7FFFFF00LL) return SLIM_ERR_UNSUPPORTED;   // the kernel indexes rows with 32-bit integers
     dim3 grid((unsigned)blocks, (unsigned)B, 2);
-    slim_append_kernel<<<grid, kAppendThreads, 0, stream>>>(
+    slim_append_kernel<NV><<<grid, kAppendThreads, 0, stream>>>(
         c->codes, c->scales, c->block_table, static_cast<const __nv_bfloat16 *>(k_new),
         static_cast<const __nv_bfloat16 *>(v_new), cu_new, start_pos, c->num_kv_heads, c->max_pages_per_seq,
-        c->num_pages);
+        c->num_pages, kGroups / c->num_kv_heads, kGroups % c->num_kv_heads);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }

@@ -68,3 +68,31 @@ def dense_attention(q, k_hat, v_hat, kv_len, sm_scale):
         P = P / P.sum(axis=1, keepdims=True)
         out[:, h, :] = P @ v_hat[:kv_len, g, :]
     return out
+
+
+def mantissa_sweep_bits(exponents, offsets=range(0, 10), subnormal_amax=(1, 2, 3, 64, 127)):
+    """Rows of 128 bf16 bit patterns that sweep significands and magnitudes (inputs only, no quantiser arithmetic).
+
+    For every unbiased exponent e in `exponents`, every one of the 128 bf16 significands of the row's
+    largest element and every k in `offsets`: one row whose largest element is +-(1.m) * 2^e at position
+    m, the other positions holding all 128 significands at exponent e - k (those that would exceed the
+    largest element are set to zero), signs alternating.  Then, for the subnormal patterns given, rows
+    whose largest element is that subnormal and whose other elements are the smaller subnormals."""
+    rows = []
+    mant = np.arange(128, dtype=np.uint32)
+    sign = ((mant & 1) << 15).astype(np.uint32)
+    for e in exponents:
+        for m in range(128):
+            for k in offsets:
+                ex = e - k
+                if ex < -126:
+                    continue
+                row = (np.uint32(ex + 127) << 7) | mant | sign
+                if k == 0:
+                    row = np.where(mant > m, 0, row)
+                row[m] = (np.uint32(e + 127) << 7) | np.uint32(m) | (np.uint32((m >> 1) & 1) << 15)
+                rows.append(row.astype(np.uint16))
+    for m in subnormal_amax:
+        row = np.where(mant <= m, mant, mant % (m + 1)).astype(np.uint32) | sign
+        rows.append(row.astype(np.uint16))
+    return np.stack(rows)

@@ -14,7 +14,7 @@ import torch
 
 from oracle import slim_oracle as so
 from paper_2407_07304_b200 import workloads
-from helpers import bf16_bits
+from helpers import bf16_bits, mantissa_sweep_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -170,6 +170,23 @@ def test_scale_extremes_and_zero_rows():
         want = so.attention(bf16_bits(w.q_decode[s]), *oc[0], 151 + s, w.sm_scale)
         denom = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
         assert (np.abs(o.float().cpu().numpy() - want) / denom).max() < 2e-2
+
+
+def test_quantiser_significand_sweep_and_extreme_magnitudes():
+    # codes and scales, bit for bit, on rows that sweep every significand of the largest element against every
+    # significand of the others, 0..9 binades below it, at magnitudes from subnormal to 2^120 (the kernel rescales
+    # rows outside [2^-60, 2^60]); three kv heads, so that a thread's rows change token in the middle of a block
+    bits = mantissa_sweep_bits([-126, -120, -61, -60, 0, 60, 61, 120])
+    n = bits.shape[0] // 3 * 3
+    k = torch.from_numpy(bits[:n].view(np.int16).copy()).view(torch.bfloat16).reshape(n // 3, 3, 128)
+    v = torch.flip(k, dims=[0]).contiguous()
+    w = workloads.Workload("sweep", 0, 1, 3, 3, [0], [n // 3], 0)
+    w.k.append(k)
+    w.v.append(v)
+    from paper_2407_07304_b200 import harness
+    run = harness.LayerRun(w)
+    run.append([n // 3])
+    _assert_cache_bits(run, _oracle_cache(w))
 
 
 def test_chunked_prefill_offset_and_shuffled_pages():

@@ -7,7 +7,7 @@ import torch
 
 from oracle import slim_oracle as so
 from paper_2407_07304_b200 import workloads
-from helpers import bf16_bits, bits_to_f64, exact_codes
+from helpers import bf16_bits, bits_to_f64, exact_codes, mantissa_sweep_bits
 
 
 def _rows(seed, n, **kw):
@@ -29,6 +29,22 @@ def test_exact_rational_brute_force():
             lo, hi = np.nextafter(np.float32(s), np.float32(-np.inf)), np.nextafter(np.float32(s), np.float32(np.inf))
             err = abs(Fraction(s) - scale_fr)
             assert err <= abs(Fraction(float(lo)) - scale_fr) and err <= abs(Fraction(float(hi)) - scale_fr)
+
+
+def test_significand_sweep_and_extreme_magnitudes_against_exact_rationals():
+    # every significand of the largest element, element exponents 0..9 below it, magnitudes from subnormal
+    # to 2^120: a sample of the rows against exact Fraction arithmetic, every scale against IEEE fp32 division
+    bits = mantissa_sweep_bits([-126, -120, -61, -60, 0, 60, 61, 120])
+    codes, scales = so.quantize(bits)
+    vals = bits_to_f64(bits)
+    picked = list(range(0, bits.shape[0], 37)) + list(range(bits.shape[0] - 5, bits.shape[0]))
+    for r in picked:
+        want, _ = exact_codes(vals[r])
+        assert codes[r].tolist() == want, f"row {r}"
+    amax = np.abs(vals).max(axis=1).astype(np.float32)
+    with np.errstate(under="ignore"):
+        want_scale = amax / np.float32(127.0)
+    assert np.array_equal(scales.view(np.uint32), want_scale.view(np.uint32))
 
 
 def test_scale_bits_match_fp32_division():
