@@ -457,6 +457,47 @@ def extra_numbers(slim, workloads, dev):
         return {"workload": w.name, "tokens": n, "ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
                 "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
 
+    def batched_prefill_numbers():
+        """One slim_attn_prefill call over sixteen prompts of 256..4096 tokens (variable-length batch)."""
+        w = workloads.make_batched_prefill()
+        r = LayerRun(w, device=dev)
+        r.append(w.prefill_len)
+        cu = [0]
+        for n in w.prefill_len:
+            cu.append(cu[-1] + n)
+        cu_d = torch.tensor(cu, dtype=torch.int32, device=dev)
+        kv_d = torch.tensor(w.prefill_len, dtype=torch.int32, device=dev)
+        qb = torch.cat([t.to(dev) for t in w.q_prefill]).contiguous()
+        ob = torch.empty_like(qb)
+        mx = max(w.prefill_len)
+
+        def pf():
+            slim.slim_attn_prefill(r.cache, qb, ob, cu_d, kv_d, w.B, mx, mx, w.Hq, w.sm_scale, r.ws_prefill, stream)
+
+        ms = time_it(pf, 5)
+        fl = sum(4 * 128 * w.Hq * n * (n + 1) // 2 for n in w.prefill_len)
+        return {"workload": w.name, "tokens": cu[-1], "lengths": w.prefill_len, "ms": ms,
+                "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
+
+    def chunked_prefill_numbers(n=2048):
+        """The last n tokens of workload 3 attend over its whole 8192-token cache (q_len < kv_len)."""
+        w = workloads.make_workload(3)
+        r = LayerRun(w, device=dev)
+        r.append(w.prefill_len)
+        S_ = w.prefill_len[0]
+        cu_d = torch.tensor([0, n], dtype=torch.int32, device=dev)
+        kv_d = torch.tensor([S_], dtype=torch.int32, device=dev)
+        qc = w.q_prefill[0][S_ - n:].to(dev).contiguous()
+        oc_ = torch.empty_like(qc)
+
+        def pf():
+            slim.slim_attn_prefill(r.cache, qc, oc_, cu_d, kv_d, 1, n, S_, w.Hq, w.sm_scale, r.ws_prefill, stream)
+
+        ms = time_it(pf, 5)
+        fl = 4 * 128 * w.Hq * (n * (S_ - n) + n * (n + 1) // 2)
+        return {"workload": w.name + f"_last{n}", "q_tokens": n, "kv_tokens": S_, "ms": ms,
+                "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
+
     def step_numbers(index, label):
         """slim_decode_step (append of one token per sequence + decode in one call) at the workload's final context."""
         w = workloads.make_workload(index)
@@ -484,6 +525,8 @@ def extra_numbers(slim, workloads, dev):
                 "prefill_c1": prefill_numbers(1),
                 "step_c1": step_numbers(1, "2 MB, L2-resident: a latency number"),
                 "step_c5": step_numbers(5, "17 MB, L2-resident: a latency number"),
+                "prefill_batched": batched_prefill_numbers(),
+                "prefill_chunked": chunked_prefill_numbers(),
                 # one sequence, 32 heads, the sequence lengths of the paper's Table 3 (256 ... 4096 tokens)
                 "prefill_sweep": [prefill_numbers(3, shrink=k, reps=10) for k in (32, 16, 8, 4, 2)]}
     return {**more, **{

@@ -125,11 +125,11 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // Blocks are handed out in the order of their linear index: heads vary fastest, then row blocks from the last
-    // (which sees the most keys) to the first, so that every head's longest blocks start first and the short
-    // ones fill the tail of the launch.
-    const int qblock = p.n_qblocks - 1 - blockIdx.y;
-    const int h = blockIdx.x, b = blockIdx.z;
+    // Blocks are handed out in the order of their linear index: heads vary fastest, then sequences, then row
+    // blocks from the last (which sees the most keys) to the first, so that the longest blocks of every head and
+    // sequence start first and the short ones fill the tail of the launch.
+    const int qblock = p.n_qblocks - 1 - blockIdx.z;
+    const int h = blockIdx.x, b = blockIdx.y;
     const int q0 = p.cu_q[b];
     const int q_len = p.cu_q[b + 1] - q0;
     const int m0 = qblock * kPfRows;
@@ -587,8 +587,8 @@ int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int
     if (rc != SLIM_OK) return rc;
     rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_prefill_tc_kernel), (int)pfl::kBytes);
     if (rc != SLIM_OK) return rc;
-    if (p.n_qblocks > 65535) return SLIM_ERR_UNSUPPORTED;
-    dim3 grid((unsigned)Hq, (unsigned)p.n_qblocks, (unsigned)B);
+    if (p.n_qblocks > 65535 || B > 65535) return SLIM_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)Hq, (unsigned)B, (unsigned)p.n_qblocks);
     slim_prefill_tc_kernel<<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;

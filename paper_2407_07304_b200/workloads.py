@@ -117,6 +117,22 @@ def make_workload(index, shrink=1):
     return w
 
 
+def make_batched_prefill(shrink=1, B=16):
+    """Batched variable-length prefill in the Llama-2-7B shape (32 q = 32 kv heads): B prompts of
+    U{256..4096} tokens (integer, drawn from the seed), all attended causally in one call.  A serving-style
+    case beside the five configured workloads; shrink divides the token counts."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(SEED0 + 6)
+    lo, hi = max(1, 256 // shrink), max(1, 4096 // shrink)
+    lens = torch.randint(lo, hi + 1, (B,), generator=gen).tolist()
+    w = Workload("batched_prefill_b16_len256_4096", 6, B, 32, 32, lens, [0] * B, 0)
+    for b in range(B):
+        w.k.append(_randn_bf16(gen, (lens[b], w.Hkv, HEAD_DIM)))
+        w.v.append(_randn_bf16(gen, (lens[b], w.Hkv, HEAD_DIM)))
+    w.q_prefill = [_randn_bf16(gen, (n, w.Hq, HEAD_DIM)) for n in lens]
+    return w
+
+
 def random_rows(seed, n_rows, outlier=False, zero_rows=0):
     """bf16 [n_rows, 128] rows for quantiser tests; the first zero_rows are all zero."""
     gen = torch.Generator(device="cpu")

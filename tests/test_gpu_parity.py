@@ -117,6 +117,27 @@ def test_c3_full_sampled_rows():
     _check(workloads.make_workload(3), prefill_rows=48)
 
 
+def test_batched_ragged_prefill_full_size_sampled():
+    # sixteen prompts of 256..4096 tokens attended in one call (the case the bench times as prefill_batched)
+    _check(workloads.make_batched_prefill(), prefill_rows=6)
+
+
+def test_chunked_prefill_full_size_sampled():
+    # the last 2048 of workload 3's 8192 tokens attend over the whole cache (q_len < kv_len), as the bench's
+    # prefill_chunked case does; sampled rows against the oracle's rows 6144.. of the full causal prefill
+    from paper_2407_07304_b200 import harness
+    w = workloads.make_workload(3)
+    S, n = w.prefill_len[0], 2048
+    oc = _oracle_cache(w)
+    run = harness.LayerRun(w)
+    run.append([S])
+    _assert_cache_bits(run, oc)
+    out = run.prefill([w.q_prefill[0][S - n:]])[0]
+    sel = _sample_rows(n, 24, 5)
+    want = so.attention(bf16_bits(w.q_prefill[0]), *oc[0], S, w.sm_scale, sel=[S - n + r for r in sel])
+    _assert_close(out[torch.tensor(sel, device=out.device)], want, "chunked prefill of workload 3")
+
+
 def test_c5_full_sampled():
     _check(workloads.make_workload(5), prefill_rows=24, decode_steps={0, 31, 63})
 

@@ -37,3 +37,11 @@ def test_structure():
     assert torch.all((std > 4).sum(dim=1) == 4)
     w5 = workloads.make_workload(5, shrink=64)
     assert w5.total_len(0) == 2 * 256 and w5.decode_steps == 64
+
+
+def test_batched_prefill_workload_is_seeded_and_ragged():
+    a, b = workloads.make_batched_prefill(shrink=16), workloads.make_batched_prefill(shrink=16)
+    assert a.prefill_len == b.prefill_len and a.B == 16 and a.Hq == a.Hkv == 32
+    assert all(16 <= n <= 256 for n in a.prefill_len) and len(set(a.prefill_len)) > 8
+    assert all(torch.equal(x, y) for x, y in zip(a.k + a.v + a.q_prefill, b.k + b.v + b.q_prefill))
+    assert [t.shape[0] for t in a.q_prefill] == a.prefill_len
