@@ -370,7 +370,7 @@ def run_ours(args, rank, world, local_rank):
 
 # dram bytes read + written by one slim_decode_stream_kernel launch on this workload (281.29 MB read,
 # 5.82 MB written), from the ncu capture summarised under profiles/.
-TRAFFIC_PER_LAUNCH = 287.11e6
+TRAFFIC_PER_LAUNCH = 286.23e6
 
 
 def extra_numbers(slim, workloads, dev):
