@@ -86,6 +86,61 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
     }
 }
 
+// The same merge for rows of fewer than 32 chunks: one warp per (sequence, query head) row, a lane owns four head
+// dims, lane c owns chunk c's (m, l).  Nothing but the row's length is waited for before the partials are
+// requested: the first sixteen chunk slots of the row are read while the length is still on its way (slots past
+// the row's last chunk hold stale values, which are replaced by zeros before use), so a row costs two round trips
+// to memory instead of one per step of the reduction.
+constexpr int kMergeWarpBatch = 16;
+constexpr int kMergeWarpsPerBlock = 8;
+__global__ void __launch_bounds__(kMergeWarpsPerBlock * 32)
+slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                              const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
+                              int B, int Hq, int n_chunks, int chunk_tokens)
+{
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * kMergeWarpsPerBlock + (threadIdx.x >> 5);   // b * Hq + h
+    pdl_wait();   // the split pass before this kernel must have finished writing the partials
+    if (row >= B * Hq) return;
+    const int len = __ldg(kv_len + row / Hq);
+    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_chunks;
+    const float4 *po = reinterpret_cast<const float4 *>(part_o + (size_t)row * n_chunks * kHeadDim) + lane;
+    float4 o[kMergeWarpBatch];
+#pragma unroll
+    for (int u = 0; u < kMergeWarpBatch; ++u)
+        o[u] = (u < n_chunks) ? __ldcg(po + (size_t)u * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float2 v = (lane < n_chunks) ? __ldcg(ml + lane) : make_float2(-INFINITY, 0.f);
+    const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
+    if (lane >= nc) v = make_float2(-INFINITY, 0.f);
+    const float M = warp_max(v.x);
+    const float w = (lane < nc) ? exp2f(v.x - M) : 0.f;
+    const float l = warp_sum(v.y * w);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = 0; c0 < nc; c0 += kMergeWarpBatch) {
+        if (c0 > 0) {
+#pragma unroll
+            for (int u = 0; u < kMergeWarpBatch; ++u)
+                o[u] = (c0 + u < nc) ? __ldcg(po + (size_t)(c0 + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kMergeWarpBatch; ++u) {
+            const float wj = __shfl_sync(0xffffffffu, w, (c0 + u) & 31);
+            if (c0 + u < nc) {   // a slot past the row's last chunk may hold anything, a NaN included
+                acc.x = fmaf(o[u].x, wj, acc.x);
+                acc.y = fmaf(o[u].y, wj, acc.y);
+                acc.z = fmaf(o[u].z, wj, acc.z);
+                acc.w = fmaf(o[u].w, wj, acc.w);
+            }
+        }
+    }
+    const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<uint32_t *>(&lo);
+    packed.y = *reinterpret_cast<uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(out + (size_t)row * kHeadDim + lane * 4) = packed;
+}
+
 // ---------------------------------------------------------------- host side
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv)
 {
@@ -168,8 +223,10 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
         SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, (const float *)p.part_o,
                                  (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
     } else {
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<1>, dim3(rows), dim3(kHeadDim), 0, stream, (const float *)p.part_o,
-                                 (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
+        const int blocks = (rows + kMergeWarpsPerBlock - 1) / kMergeWarpsPerBlock;
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_warp_kernel, dim3(blocks), dim3(kMergeWarpsPerBlock * 32), 0, stream,
+                                 (const float *)p.part_o, (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq,
+                                 p.n_chunks, C));
     }
     return SLIM_OK;
 }
