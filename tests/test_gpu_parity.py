@@ -168,6 +168,23 @@ def test_group_sizes(Hq, Hkv):
     _check(_custom(2, Hq, Hkv, [70, 200], [37, 0], 2, 200 + Hq))
 
 
+def test_random_shapes_against_the_oracle():
+    # sixty seeded random problems: batch 1..5, 1..8 kv heads, 1..16 query heads per kv head, prompt lengths at and
+    # around the 128-token page and 256-token chunk boundaries, a bulk append, up to three decode steps (as
+    # append + decode or as one call); every code, scale and output is compared
+    import random
+    rng = random.Random(20240707)
+    for _ in range(60):
+        B = rng.randint(1, 5)
+        Hkv = rng.choice([1, 2, 3, 4, 8])
+        G = rng.choice([1, 1, 2, 4, 8, 16])
+        pre = [rng.choice([1, 2, 127, 128, 129, 255, 256, 257, 300, 511, 513, rng.randint(1, 1200)]) for _ in range(B)]
+        bulk = [rng.choice([0, 0, 1, 130, rng.randint(0, 600)]) for _ in range(B)]
+        steps = rng.choice([0, 1, 2, 3])
+        one = steps > 0 and rng.random() < 0.5
+        _check(_custom(B, Hkv * G, Hkv, pre, bulk, steps, rng.randint(0, 10 ** 6)), one_call_step=one)
+
+
 def test_scale_extremes_and_zero_rows():
     # rows scaled far apart, zero K and V rows, and large-magnitude queries
     w = _custom(1, 2, 1, [150], [0], 2, 300)
