@@ -439,7 +439,7 @@ def extra_numbers(slim, workloads, dev):
         return {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
                 "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "cache": label}
 
-    def prefill_numbers(index, shrink=1, reps=3):
+    def prefill_numbers(index, shrink=1, reps=3, two_pass=False):
         w = workloads.make_workload(index, shrink=shrink)
         r = LayerRun(w, device=dev)
         n = w.prefill_len[0]
@@ -449,11 +449,13 @@ def extra_numbers(slim, workloads, dev):
         q5 = w.q_prefill[0].to(dev).contiguous()
         o5 = torch.empty_like(q5)
 
+        call = slim.slim_attn_prefill_two_pass if two_pass else slim.slim_attn_prefill
+
         def pf():
-            slim.slim_attn_prefill(r.cache, q5, o5, cu5, kv5, 1, n, n, w.Hq, w.sm_scale, r.ws_prefill, stream)
+            call(r.cache, q5, o5, cu5, kv5, 1, n, n, w.Hq, w.sm_scale, r.ws_prefill, stream)
 
         ms = time_it(pf, reps)
-        fl = 4 * 128 * w.Hq * n * (n + 1) // 2
+        fl = 4 * 128 * w.Hq * n * (n + 1) // 2   # the attention's flops: the second Q.K^T of the two-pass form is not counted
         return {"workload": w.name, "tokens": n, "ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
                 "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
 
@@ -525,6 +527,9 @@ def extra_numbers(slim, workloads, dev):
                 "prefill_c1": prefill_numbers(1),
                 "step_c1": step_numbers(1, "2 MB, L2-resident: a latency number"),
                 "step_c5": step_numbers(5, "17 MB, L2-resident: a latency number"),
+                # the literal order (all scores of a row, then softmax, then .V): maxima first, no corrections
+                "prefill_two_pass_c3": prefill_numbers(3, two_pass=True),
+                "prefill_two_pass_sweep": [prefill_numbers(3, shrink=k, reps=10, two_pass=True) for k in (32, 16, 8, 4, 2)],
                 "prefill_batched": batched_prefill_numbers(),
                 "prefill_chunked": chunked_prefill_numbers(),
                 # one sequence, 32 heads, the sequence lengths of the paper's Table 3 (256 ... 4096 tokens)

@@ -127,6 +127,21 @@ int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out,
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same attention in the literal order of Section 2.1: every score of a
+ * query row is formed before its softmax.  The kernel walks a row block's keys
+ * twice - first the row maxima of the scores, then P = exp(s - max) against
+ * the final maximum and P.V - so no partial result is ever corrected.  It
+ * forms Q.K^T twice and is therefore slower than slim_attn_prefill, which
+ * streams the keys once behind a running maximum; it exists to measure that
+ * difference.  Arguments, layout, workspace and error behaviour are those of
+ * slim_attn_prefill; the two results agree within the output tolerance.
+ */
+int slim_attn_prefill_two_pass(const slim_cache_t *cache, const void *q, void *out,
+                               const int32_t *cu_q, const int32_t *kv_len,
+                               int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq, float sm_scale,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Decode attention: one query token per sequence against all kv_len[b] cached
  * tokens (the new token's K/V already appended).  Same arithmetic as above with
  * q_len == 1.  The next-token phase is a matrix-vector product bound by memory

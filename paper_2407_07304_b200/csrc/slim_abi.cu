@@ -24,7 +24,7 @@ int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const
                   const int32_t *kv_len, int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
-                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
+                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass);
 size_t prefill_workspace_bytes();
 
 static int check_cache(const slim_cache_t *c)
@@ -55,9 +55,9 @@ SLIM_EXPORT int slim_kv_append(const slim_cache_t *cache, const void *k_new, con
     return launch_append(cache, k_new, v_new, cu_new, start_pos, B, max_new, (cudaStream_t)stream);
 }
 
-SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
-                                  const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
-                                  float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
+static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
+                         const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
+                         float sm_scale, void *workspace, size_t workspace_bytes, void *stream, bool two_pass)
 {
     int rc = check_cache(cache);
     if (rc != SLIM_OK) return rc;
@@ -70,7 +70,21 @@ SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void
     if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
     const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
-    return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream);
+    return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream, two_pass);
+}
+
+SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
+                                  const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
+                                  float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, false);
+}
+
+SLIM_EXPORT int slim_attn_prefill_two_pass(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
+                                           const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
+                                           float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, true);
 }
 
 // Shared validation of the decode entry points; *launch is false for a valid no-op.

@@ -120,6 +120,12 @@ __device__ __forceinline__ uint32_t pf_hmul2(uint32_t a, uint32_t b)
     return r;
 }
 
+// kTwoPass: the literal order of Section 2.1 - every score of a row before its softmax.  The block walks its key
+// tiles twice: the first pass only takes the row maxima of the scores, the second computes P = 2^(s - max) against
+// that final maximum and accumulates P.V, so no accumulator is ever corrected.  Both passes run through the same
+// pipeline (a key tile is loaded and converted again in the second pass); the tile sequence of the block is
+// simply twice as long, and barrier phases count positions in that sequence.
+template <bool kTwoPass>
 __global__ void __launch_bounds__(kPfThreads, 1)
 slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const PrefillTcParams p)
 {
@@ -146,6 +152,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     }
     const int T0 = Tt[0], T1 = Tt[1];
     const int T = max(T0, T1);
+    const int NT = kTwoPass ? 2 * T : T;   // positions in the block's tile sequence
     const int head = h / p.G;
 
     const uint32_t sbase = smem_u32(smem);
@@ -165,7 +172,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         const int slot = i % kPfRawStages, j = i >> 1;
         const int kv = i & 1;
         int page = page_next;
-        if (kv == 1 && j + 1 < T) page_next = __ldg(bt + j + 1);   // requested one tile ahead
+        if (kv == 1 && j + 1 < NT) page_next = __ldg(bt + ((kTwoPass && j + 1 >= T) ? j + 1 - T : j + 1));   // requested one tile ahead
         page = (page >= 0 && page < p.num_pages) ? page : 0;
         const uint32_t dst = sbase + pfl::kRaw + slot * pfl::kRawStage;
         const uint32_t full = bar(pfl::RAW_FULL, slot);
@@ -179,7 +186,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         tc::mbar_init_fence();
         if (T > 0) {
             page_next = __ldg(p.block_table + (size_t)b * p.max_pages_per_seq);
-            for (int i = 0; i < min(kPfRawStages, 2 * T); ++i) request_raw(i);   // every stage is free the first time round
+            for (int i = 0; i < min(kPfRawStages, 2 * NT); ++i) request_raw(i);   // every stage is free the first time round
         }
     }
     // Query rows are read coalesced: sixteen lanes read one row's 256 bytes, so a warp's load covers two whole rows
@@ -287,14 +294,18 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
         }
 
         float m_run = -INFINITY, l_run = 0.f;
-        for (int j = 0; j < Tmine; ++j) {
-            wait(bar(pfl::S_FULL, t), (uint32_t)j & 1u);
+        const int steps = kTwoPass ? 2 * Tmine : Tmine;   // this query tile's steps (its count of S_FULL / P_FULL / O_DONE phases)
+        for (int jj = 0; jj < steps; ++jj) {
+            const bool second = kTwoPass && jj >= Tmine;
+            const int j = second ? jj - Tmine : jj;       // key tile
+            const int jv = second ? T + j : j;            // its position in the block's tile sequence
+            wait(bar(pfl::S_FULL, t), (uint32_t)jj & 1u);
             __syncwarp();   // the wait loop may leave the lanes diverged; the tensor-memory ops below are warp-aligned
             tc::fence_after_sync();
-            wait(bar(pfl::VEXP_FULL, j & 1), (uint32_t)(j >> 1) & 1u);   // published long before, as a rule
-            const float c = fmaxf(rs * misc_f[j & 1], 1e-37f);   // row scale * kexp of this key tile (> 0)
-            const float F = misc_f[2 + (j & 1)];                 // log2 vexp
-            const float vinv = misc_f[12 + (j & 1)];             // 1 / vexp
+            wait(bar(pfl::VEXP_FULL, jv & 1), (uint32_t)(jv >> 1) & 1u);   // published long before, as a rule
+            const float c = fmaxf(rs * misc_f[jv & 1], 1e-37f);   // row scale * kexp of this key tile (> 0)
+            const float F = misc_f[2 + (jv & 1)];                 // log2 vexp
+            const float vinv = misc_f[12 + (jv & 1)];             // 1 / vexp
             const int key0 = j * kPfBN;
             const bool diag = key0 + kPfBN - 1 > last_key;       // some of this tile's keys are masked for this row
             // ---- the whole score row into registers with one round trip to tensor memory, then its maximum
@@ -325,9 +336,17 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             }
             mx = fmaxf(mx, mx2);
             const float mt = (mx == -INFINITY) ? -INFINITY : fmaf(mx, c, F);   // the tile's largest s'
+            if (kTwoPass && !second) {
+                // first pass: the row's maximum only; the score buffer is free for the next tile's scores
+                m_run = fmaxf(m_run, mt);
+                tc::fence_before_sync();
+                tc::mbar_arrive(bar(pfl::P_FULL, t));
+                continue;
+            }
             // the reference maximum only moves when the tile's exceeds it by more than the threshold
-            const bool grow = (j == 0) ? true : (mt > m_run + kPfRescaleThreshold);
-            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+            // (second pass of the two-pass form: it is the row's final maximum and never moves)
+            const bool grow = kTwoPass ? false : ((j == 0) ? true : (mt > m_run + kPfRescaleThreshold));
+            if (!kTwoPass && j > 0 && __any_sync(0xffffffffu, grow)) {
                 const float alpha = grow ? pf_exp2(m_run - mt) : 1.f;   // m_run = -inf gives 0
                 wait(bar(pfl::O_DONE, t), (uint32_t)(j - 1) & 1u);      // P.V of the previous tile is complete
                 __syncwarp();
@@ -375,7 +394,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
 
         // ---- epilogue: O / l -> bf16
         if (Tmine > 0) {
-            wait(bar(pfl::O_DONE, t), (uint32_t)(Tmine - 1) & 1u);
+            wait(bar(pfl::O_DONE, t), (uint32_t)(steps - 1) & 1u);
             __syncwarp();
             tc::fence_after_sync();
             const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
@@ -420,13 +439,13 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     } else if (warp < 12) {
         // =========================================================== dequantise: thread = token row of the tile
         const int r = tid - 256, cw = warp - 8;
-        for (int i = 0; i < 2 * T; ++i) {
-            const int slot = i % kPfRawStages, j = i >> 1;
+        for (int i = 0; i < 2 * NT; ++i) {
+            const int slot = i % kPfRawStages, j = i >> 1;   // j: position in the block's tile sequence
             const bool is_k = (i & 1) == 0;   // K tile first, then the V tile of the same keys
             wait(bar(pfl::RAW_FULL, slot), (uint32_t)(i / kPfRawStages) & 1u);
             if (is_k) wait(bar(pfl::KF_EMPTY, 0), ((uint32_t)j & 1u) ^ 1u);
             const unsigned char *raw = smem + pfl::kRaw + slot * pfl::kRawStage;
-            const int n_valid = min(kPfBN, kvl - j * kPfBN);   // rows past the cache length hold anything: zeroed
+            const int n_valid = min(kPfBN, kvl - ((kTwoPass && j >= T) ? j - T : j) * kPfBN);   // rows past the cache length hold anything: zeroed
             const float sc = (r < n_valid) ? reinterpret_cast<const float *>(raw + 16384)[r] : 0.f;
             // power of two below the tile's largest scale; the exchange buffers alternate with j so that a fast
             // warp cannot overwrite what a slow one still reads
@@ -474,7 +493,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     } else if (warp == 12) {
         // =========================================================== loader (one thread)
         if (lane == 0 && T > 0) {
-            for (int i = kPfRawStages; i < 2 * T; ++i) {   // the first round of the ring was requested during set-up
+            for (int i = kPfRawStages; i < 2 * NT; ++i) {   // the first round of the ring was requested during set-up
                 wait(bar(pfl::RAW_EMPTY, i % kPfRawStages), ((uint32_t)(i / kPfRawStages) & 1u) ^ 1u);
                 request_raw(i);
             }
@@ -516,14 +535,21 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             tc::commit(bar(pfl::KF_EMPTY, 0));
             // The fixed order P0.V(j), Q0.K(j+1)^T, P1.V(j), Q1.K(j+1)^T keeps the two query tiles half a step
             // apart, so that their softmax phases (which share the special-function units) alternate.
-            for (int j = 0; j < T; ++j) {
-                const uint32_t ph = (uint32_t)j & 1u, phn = ph ^ 1u;
-                const bool a0 = j < T0, a1 = j < T1, n0 = j + 1 < T0, n1 = j + 1 < T1;
+            int c0 = 0, c1 = 0;   // two-pass form: steps each query tile has taken (its barrier phases)
+            for (int jv = 0; jv < NT; ++jv) {
+                const uint32_t ph = (uint32_t)jv & 1u, phn = ph ^ 1u;
+                const bool second = kTwoPass && jv >= T;
+                const int j = second ? jv - T : jv;                          // key tile at this position
+                const int jn = (kTwoPass && jv + 1 >= T) ? jv + 1 - T : jv + 1;   // key tile at the next position
+                const bool more = jv + 1 < NT;
+                const bool a0 = j < T0, a1 = j < T1, n0 = more && jn < T0, n1 = more && jn < T1;
+                const bool pv = !kTwoPass || second;                         // the first pass has no P.V
                 wait(bar(pfl::VF_FULL, 0), ph);
                 if (a0) {
-                    wait(bar(pfl::P_FULL, 0), ph);
+                    wait(bar(pfl::P_FULL, 0), kTwoPass ? ((uint32_t)c0 & 1u) : ph);
                     tc::fence_after_sync();
-                    issue_pv(0, j == 0);
+                    if (pv) issue_pv(0, j == 0); else tc::commit(bar(pfl::O_DONE, 0));
+                    ++c0;
                 }
                 if (n0 || n1) wait(bar(pfl::KF_FULL, 0), phn);
                 if (n0) {
@@ -531,9 +557,10 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                     issue_qk(0);
                 }
                 if (a1) {
-                    wait(bar(pfl::P_FULL, 1), ph);
+                    wait(bar(pfl::P_FULL, 1), kTwoPass ? ((uint32_t)c1 & 1u) : ph);
                     tc::fence_after_sync();
-                    issue_pv(1, j == 0);
+                    if (pv) issue_pv(1, j == 0); else tc::commit(bar(pfl::O_DONE, 1));
+                    ++c1;
                 }
                 tc::commit(bar(pfl::VF_EMPTY, 0));
                 if (n1) {
@@ -564,7 +591,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
 size_t prefill_workspace_bytes() { return 16; }   // status word
 
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
-                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream)
+                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass)
 {
     PrefillTcParams p;
     p.scales = c->scales;
@@ -585,11 +612,13 @@ int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int
     CUtensorMap map;
     int rc = codes_tensor_map(c, kPfBN, &map);
     if (rc != SLIM_OK) return rc;
-    rc = allow_dynamic_smem(reinterpret_cast<const void *>(slim_prefill_tc_kernel), (int)pfl::kBytes);
+    rc = allow_dynamic_smem(two_pass ? reinterpret_cast<const void *>(slim_prefill_tc_kernel<true>)
+                                     : reinterpret_cast<const void *>(slim_prefill_tc_kernel<false>), (int)pfl::kBytes);
     if (rc != SLIM_OK) return rc;
     if (p.n_qblocks > 65535 || B > 65535) return SLIM_ERR_UNSUPPORTED;
     dim3 grid((unsigned)Hq, (unsigned)B, (unsigned)p.n_qblocks);
-    slim_prefill_tc_kernel<<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
+    if (two_pass) slim_prefill_tc_kernel<true><<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
+    else slim_prefill_tc_kernel<false><<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }

@@ -138,6 +138,54 @@ def test_chunked_prefill_full_size_sampled():
     _assert_close(out[torch.tensor(sel, device=out.device)], want, "chunked prefill of workload 3")
 
 
+def _check_two_pass(w, prefill_rows=None):
+    """slim_attn_prefill_two_pass (maxima first, then P.V) against the oracle, and against the one-pass kernel."""
+    from paper_2407_07304_b200 import binding as slim, harness
+    oc = _oracle_cache(w)
+    run = harness.LayerRun(w)
+    run.append(w.prefill_len)
+    out = run.prefill(w.q_prefill, two_pass=True)
+    ref = run.prefill(w.q_prefill)
+    torch.cuda.synchronize()
+    assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
+    for b in range(w.B):
+        n = w.prefill_len[b]
+        sel = None if prefill_rows is None else _sample_rows(n, prefill_rows, 23 + b)
+        want = so.attention(bf16_bits(w.q_prefill[b]), *oc[b], n, w.sm_scale, sel=sel)
+        idx = slice(None) if sel is None else torch.tensor(sel, device=out[b].device)
+        _assert_close(out[b][idx], want, f"{w.name} two-pass prefill seq {b}")
+        # both kernels round the same exact result: they differ by a few bf16 ulps at most
+        d = (out[b].float() - ref[b].float()).abs().max().item()
+        assert d <= 2 * MAX_ABS, f"{w.name} seq {b}: two-pass and one-pass outputs differ by {d}"
+
+
+@pytest.mark.parametrize("index,shrink", [(1, 1), (3, 16), (5, 32)])
+def test_two_pass_prefill_small_all_outputs(index, shrink):
+    _check_two_pass(workloads.make_workload(index, shrink=shrink))
+
+
+@pytest.mark.parametrize("lens", [[1], [2, 127], [128, 129], [255, 256, 257], [1, 383, 640]])
+def test_two_pass_prefill_ragged_lengths(lens):
+    B = len(lens)
+    _check_two_pass(_custom(B, 4, 2, lens, [0] * B, 0, 700 + lens[0]))
+
+
+def test_two_pass_prefill_with_cached_prefix():
+    # q_len < kv_len: the last 70 of 330 cached tokens attend
+    from paper_2407_07304_b200 import harness
+    w = _custom(1, 8, 2, [330], [0], 0, 900)
+    oc = _oracle_cache(w)
+    run = harness.LayerRun(w)
+    run.append([330])
+    out = run.prefill([w.q_prefill[0][260:]], two_pass=True)[0]
+    want = so.attention(bf16_bits(w.q_prefill[0]), *oc[0], 330, w.sm_scale, sel=list(range(260, 330)))
+    _assert_close(out, want, "two-pass prefill behind a cached prefix")
+
+
+def test_two_pass_prefill_c3_full_sampled_rows():
+    _check_two_pass(workloads.make_workload(3), prefill_rows=24)
+
+
 def test_c5_full_sampled():
     _check(workloads.make_workload(5), prefill_rows=24, decode_steps={0, 31, 63})
 
