@@ -548,7 +548,9 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 int last = nc - 1 - range[3];   // list index of the pair's last chunk
                 const int kv = lane >> 4, l = lane & 15;
                 for (int r = 0; last < cnt; ++r) {
-                    if (r % kPW == warp) {
+                    // dealt from the last consumer warp down: the first group, which takes the block's first chunk,
+                    // gets a row only when a block owns more than eight new tokens
+                    if (kPW - 1 - r % kPW == warp) {
                         const int pos = len - 1;
                         // a length beyond the page table or the launch's max_kv was clamped: its token has no slot
                         const bool has_slot = __ldg(p.kv_len + b) == len;
