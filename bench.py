@@ -516,11 +516,31 @@ def extra_numbers(slim, workloads, dev):
             slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, stream)
 
         ms = time_it(st, 50)
-        return {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "cache": label}
+        # the same step replayed from a CUDA graph of twenty calls: the device-side latency of a step without the
+        # host's launch cost between steps (the same new row goes to the same slot every time: idempotent)
+        side = torch.cuda.Stream()
+        n_in_graph = 20
+        with torch.cuda.stream(side):
+            slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, side)
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
+                for _ in range(n_in_graph):
+                    slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, side)
+            g.replay()
+            side.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            for _ in range(5):
+                g.replay()
+            e1.record(side)
+            side.synchronize()
+            ms_graph = e0.elapsed_time(e1) / (5 * n_in_graph)
+        return {"workload": w.name, "ms": ms, "ms_graph_replay": ms_graph, "tokens_per_s": w.B / (ms * 1e-3), "cache": label}
 
     more = {}
     if not os.environ.get("SLIM_BENCH_SHORT"):
-        more = {"decode_c4": decode_numbers(4, 2, "two cache copies rotated (2 x 173 MB > L2)"),
+        more = {"decode_c4": decode_numbers(4, 2, "two cache copies rotated (2 x 187 MB > L2)"),
                 "decode_c5": decode_numbers(5, 1, "17 MB, L2-resident: a latency number, not an HBM number"),
                 "decode_c1": decode_numbers(1, 1, "2 MB, L2-resident: a latency number, not an HBM number"),
                 "prefill_c5": prefill_numbers(5),
