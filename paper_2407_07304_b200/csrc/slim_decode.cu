@@ -86,6 +86,15 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
     }
 }
 
+// A 16-byte load past the L1 cache that the compiler keeps where it is written (the merge kernels request a
+// row's partials before the values that decide which of them count have arrived).
+__device__ __forceinline__ float4 ld_cg_now(const float4 *ptr)
+{
+    float4 v;
+    asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr) : "memory");
+    return v;
+}
+
 // The same merge for rows of fewer than 32 chunks: one warp per (sequence, query head) row, a lane owns four head
 // dims, lane c owns chunk c's (m, l).  Nothing but the row's length is waited for before the partials are
 // requested: the first sixteen chunk slots of the row are read while the length is still on its way (slots past
@@ -139,6 +148,77 @@ slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__r
     packed.x = *reinterpret_cast<uint32_t *>(&lo);
     packed.y = *reinterpret_cast<uint32_t *>(&hi);
     *reinterpret_cast<uint2 *>(out + (size_t)row * kHeadDim + lane * 4) = packed;
+}
+
+// Rows of 32 to 16 * kWarps chunks: one block per row, warp w owns the sixteen chunk slots [16 w, 16 w + 16) and
+// merges them as the kernel above does - all of its partials requested at once, before the row's length is known -
+// into (M_w, l_w, o_w); the warps' results are then merged by the same identity through shared memory.
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32)
+slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                               const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
+                               int B, int Hq, int n_chunks, int chunk_tokens)
+{
+    __shared__ float4 acc_s[kWarps][32];
+    __shared__ float m_s[kWarps], l_s[kWarps];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int row = blockIdx.x;   // b * Hq + h
+    pdl_wait();   // the split pass before this kernel must have finished writing the partials
+    const int len = __ldg(kv_len + row / Hq);
+    const int c_base = w * kMergeWarpBatch;
+    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_chunks;
+    const float4 *po = reinterpret_cast<const float4 *>(part_o + (size_t)row * n_chunks * kHeadDim) + lane;
+    float4 o[kMergeWarpBatch];
+#pragma unroll
+    for (int u = 0; u < kMergeWarpBatch; ++u)
+        o[u] = (c_base + u < n_chunks) ? ld_cg_now(po + (size_t)(c_base + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float2 v = (lane < kMergeWarpBatch && c_base + lane < n_chunks) ? __ldcg(ml + c_base + lane) : make_float2(-INFINITY, 0.f);
+    const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
+    const bool mine = lane < kMergeWarpBatch && c_base + lane < nc;
+    if (!mine) v = make_float2(-INFINITY, 0.f);
+    const float Mw = warp_max(v.x);
+    const float wgt = mine ? exp2f(v.x - Mw) : 0.f;
+    const float lw = warp_sum(v.y * wgt);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < kMergeWarpBatch; ++u) {
+        const float wj = __shfl_sync(0xffffffffu, wgt, u);
+        if (c_base + u < nc) {   // a slot past the row's last chunk may hold anything, a NaN included
+            acc.x = fmaf(o[u].x, wj, acc.x);
+            acc.y = fmaf(o[u].y, wj, acc.y);
+            acc.z = fmaf(o[u].z, wj, acc.z);
+            acc.w = fmaf(o[u].w, wj, acc.w);
+        }
+    }
+    acc_s[w][lane] = acc;
+    if (lane == 0) {
+        m_s[w] = Mw;   // minus infinity for a warp whose slots lie past the row's last chunk
+        l_s[w] = lw;
+    }
+    __syncthreads();
+    if (w == 0) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) M = fmaxf(M, m_s[i]);
+        float l = 0.f;
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) {
+            const float f = (m_s[i] == -INFINITY) ? 0.f : exp2f(m_s[i] - M);
+            const float4 a = acc_s[i][lane];
+            l = fmaf(l_s[i], f, l);
+            r.x = fmaf(a.x, f, r.x);
+            r.y = fmaf(a.y, f, r.y);
+            r.z = fmaf(a.z, f, r.z);
+            r.w = fmaf(a.w, f, r.w);
+        }
+        const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(r.x * inv, r.y * inv), hi = __floats2bfloat162_rn(r.z * inv, r.w * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<uint32_t *>(&lo);
+        packed.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(out + (size_t)row * kHeadDim + lane * 4) = packed;
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -219,7 +299,16 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
     int C;
     const DecodeParams p = make_params(c, nullptr, kv_len, B, max_kv, Hq, 1.f, const_cast<void *>(workspace), C);
     const int rows = B * Hq;
-    if (p.n_chunks >= 32) {
+    if (p.n_chunks >= 32 && p.n_chunks <= 16 * kMergeWarpBatch) {
+        const float *po = p.part_o, *pm = p.part_ml;
+        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(out);
+        if (p.n_chunks <= 4 * kMergeWarpBatch)
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<4>, dim3(rows), dim3(128), 0, stream, po, pm, kv_len, o, B, Hq, p.n_chunks, C));
+        else if (p.n_chunks <= 8 * kMergeWarpBatch)
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<8>, dim3(rows), dim3(256), 0, stream, po, pm, kv_len, o, B, Hq, p.n_chunks, C));
+        else
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<16>, dim3(rows), dim3(512), 0, stream, po, pm, kv_len, o, B, Hq, p.n_chunks, C));
+    } else if (p.n_chunks >= 32) {
         SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, (const float *)p.part_o,
                                  (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
     } else {

@@ -233,6 +233,13 @@ def test_random_shapes_against_the_oracle():
         _check(_custom(B, Hkv * G, Hkv, pre, bulk, steps, rng.randint(0, 10 ** 6)), one_call_step=one)
 
 
+@pytest.mark.parametrize("length", [8200, 12345, 20000, 40001, 66000])
+def test_decode_long_rows_every_merge_kernel(length):
+    # one sequence, two query heads on one kv head: 33 / 49 / 79 / 157 / 258 chunks per row, i.e. the block-per-row
+    # merge with 4, 4, 8 and 16 warps and, past 256 chunks, the four-group kernel
+    _check(_custom(1, 2, 1, [0], [length - 1], 1, 3000 + length))
+
+
 def test_scale_extremes_and_zero_rows():
     # rows scaled far apart, zero K and V rows, and large-magnitude queries
     w = _custom(1, 2, 1, [150], [0], 2, 300)
