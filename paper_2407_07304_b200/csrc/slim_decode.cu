@@ -154,7 +154,7 @@ slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__r
 // merges them as the kernel above does - all of its partials requested at once, before the row's length is known -
 // into (M_w, l_w, o_w); the warps' results are then merged by the same identity through shared memory.
 template <int kWarps>
-__global__ void __launch_bounds__(kWarps * 32)
+__global__ void __launch_bounds__(kWarps * 32, 1)
 slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                                const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
                                int B, int Hq, int n_chunks, int chunk_tokens)
@@ -171,7 +171,7 @@ slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__
     float4 o[kMergeWarpBatch];
 #pragma unroll
     for (int u = 0; u < kMergeWarpBatch; ++u)
-        o[u] = (c_base + u < n_chunks) ? ld_cg_now(po + (size_t)(c_base + u) * (kHeadDim / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        o[u] = ld_cg_now(po + (size_t)min(c_base + u, n_chunks - 1) * (kHeadDim / 4));   // n_chunks >= 32 here; slots past nc are not used
     float2 v = (lane < kMergeWarpBatch && c_base + lane < n_chunks) ? __ldcg(ml + c_base + lane) : make_float2(-INFINITY, 0.f);
     const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
     const bool mine = lane < kMergeWarpBatch && c_base + lane < nc;
