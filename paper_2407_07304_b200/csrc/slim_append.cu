@@ -1,39 +1,28 @@
 // Quantise-and-append kernel: the write side of the INT8 KV cache (Section 2.2).
 //
-// The kernel is bound by memory traffic (256 bytes read, 132 written per row), so it is laid out to
-// keep many 16-byte loads in flight per thread and to spend few instructions per element:
+// The kernel is bound by memory traffic (256 bytes read, 132 written per row), so it spends few instructions
+// per element and keeps the occupancy an HBM stream needs:
 //
 //  * 16 / NV lanes own one row (a lane holds NV pieces of eight consecutive dims: a 16-byte load and an
-//    8-byte store of codes each); a block of 256 threads handles 64 * NV consecutive rows, four per group
-//    of lanes, all loads issued before any arithmetic.
+//    8-byte store of codes each), so the per-row work - the shuffle reduction of the maximum, the reciprocal,
+//    the scale, token / head / page arithmetic - is shared by 8 NV values per lane.  NV = 4 and one row in
+//    flight per group of lanes measured fastest (33 registers, seven blocks of 256 threads per SM); more rows
+//    in flight, or 2 / 8 / 16 lanes per row, were 4 to 35 us slower on an 8192-token append.
 //  * the row quantiser itself (exact round-half-even codes, bit for bit reproducible) is in slim_quant.cuh.
 #include "slim_common.cuh"
 #include "slim_quant.cuh"
 
 namespace slim {
 
-#ifndef SLIM_APPEND_NV
-#define SLIM_APPEND_NV 4   // four lanes per row: the per-row work (shuffles, reciprocal, addresses) is shared by 32 values per lane
-#endif
-#ifndef SLIM_APPEND_ROWS
-#define SLIM_APPEND_ROWS 1
-#endif
-#ifndef SLIM_APPEND_THREADS
-#define SLIM_APPEND_THREADS 256
-#endif
-#ifdef SLIM_APPEND_MINBLOCKS
-#define SLIM_APPEND_BOUNDS __launch_bounds__(SLIM_APPEND_THREADS, SLIM_APPEND_MINBLOCKS)
-#else
-#define SLIM_APPEND_BOUNDS __launch_bounds__(SLIM_APPEND_THREADS)
-#endif
-constexpr int kAppendThreads = SLIM_APPEND_THREADS;
-constexpr int kAppendRowsPerGroup = SLIM_APPEND_ROWS;   // rows in flight per group of lanes
+constexpr int kAppendNV = 4;               // 16-byte loads per lane and row: four lanes own a row
+constexpr int kAppendThreads = 256;
+constexpr int kAppendRowsPerGroup = 1;     // rows in flight per group of lanes
 
 // NV = 16-byte loads per lane and row: 16 / NV lanes own a row.
 // grid = (ceil(max_new * Hkv / rows per block), B, 2 [K, V]); row index = token * Hkv + head within the
 // sequence's new rows.  step_tok / step_head = quotient and remainder of the block's group count by Hkv.
 template <int NV>
-__global__ void SLIM_APPEND_BOUNDS
+__global__ void __launch_bounds__(kAppendThreads)
 slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
                    const int32_t *__restrict__ block_table,
                    const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
@@ -99,7 +88,7 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
 int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
                   const int32_t *start_pos, int B, int max_new, cudaStream_t stream)
 {
-    constexpr int NV = SLIM_APPEND_NV;
+    constexpr int NV = kAppendNV;
     constexpr int kGroups = kAppendThreads / (16 / NV), kRowsPerBlock = kGroups * kAppendRowsPerGroup;
     const long long rows = (long long)max_new * c->num_kv_heads;
     const long long blocks = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
