@@ -79,7 +79,7 @@ typedef struct slim_cache {
 
 /*
  * Quantise new K and V rows and write them into the cache (Section 2.2: INT8
- * codes, "a unique scale for each token and each head").
+ * codes, one scale per (token, kv head), K and V separately).
  *
  * For each row x (128 bf16 values of one token and one kv head, K and V
  * separately): amax = max|x_d|; scale = amax / 127 (fp32, correctly rounded);
@@ -104,6 +104,14 @@ int slim_kv_append(const slim_cache_t *cache, const void *k_new, const void *v_n
 /*
  * Causal prefill attention over the INT8 cache (Section 2.1).  The new tokens'
  * K/V must already be in the cache (slim_kv_append first).
+ *
+ * This is the streamed form: a block of query rows owns every key it sees (the
+ * one-dimensional decomposition of Section 2.1, no key split and no merge
+ * between blocks), but 128-key tiles pass through the on-chip score buffer once,
+ * behind a running row maximum, instead of the whole score row being formed
+ * before its softmax.  The result is the same softmax attention; the order of
+ * Section 2.1 itself is slim_attn_prefill_two_pass (any length) and
+ * slim_attn_prefill_full_row (rows that see at most 256 keys).
  *
  * For sequence b with q_len = cu_q[b+1]-cu_q[b] query rows and kv_len[b] cached
  * tokens, query row t (0-based) sees keys j <= kv_len[b] - q_len + t; query
@@ -268,12 +276,30 @@ size_t slim_step_staging_bytes(int32_t B, int32_t Hq, int32_t Hkv);
  *    on the array and give wrong results; keep calls on one stream or order
  *    them with events.
  *
+ *  - The array's header (the status word of the bounded waits and the counters
+ *    of the in-kernel merge) cannot be reached through slim_read_status or a
+ *    memset, because the caller has no pointer to it.  slim_static_status does
+ *    what slim_read_status does for a workspace (synchronises `stream`, returns
+ *    SLIM_OK or SLIM_ERR_TIMEOUT); slim_static_reset enqueues a clear of the
+ *    header on `stream` (one cudaMemsetAsync, nothing allocated) and must
+ *    follow a SLIM_ERR_TIMEOUT before the next slim_attn_decode_static on that
+ *    device, exactly as a workspace's header must be zeroed again: a kernel
+ *    that gave up may have left counters non-zero, and later calls would then
+ *    leave rows unwritten.  slim_static_selftest_timeout is
+ *    slim_selftest_timeout aimed at the array's status word, so the sequence
+ *    timeout -> status -> reset can be exercised without any fault.
+ *  - The first of these four calls on a device performs the address lookup;
+ *    host threads may make it concurrently.
+ *
  * Arguments as for slim_attn_decode, minus the workspace.
  */
 #define SLIM_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
 int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
                             const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
                             void *stream);
+int slim_static_status(void *stream);
+int slim_static_reset(void *stream);
+int slim_static_selftest_timeout(void *stream);
 
 /*
  * Device-side waits are bounded.  The attention kernels wait on hardware barriers (TMA copies, tensor-core

@@ -7,8 +7,8 @@
  * no code with the CUDA path and nothing in the product may call it.
  *
  * What it follows:
- *   - Quantiser: the paper's "INT8 KV cache" with "a unique scale for each
- *     token and each head" (Section 2.2).  The paper gives no formula; the
+ *   - Quantiser: the INT8 KV cache of Section 2.2, one scale per (token,
+ *     kv head), K and V separately.  The paper gives no formula; the
  *     format used is symmetric codes in [-127, 127], scale = absmax / 127 kept
  *     in fp32, round half to even, evaluated on the exact ratio 127*x/absmax.
  *   - Attention: SlimAttention (Section 2.1) computes, for a block of query

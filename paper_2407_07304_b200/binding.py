@@ -25,7 +25,8 @@ PAGE_TOKENS = 128
 
 EXPORTS = (
     "slim_kv_append", "slim_attn_prefill", "slim_attn_prefill_two_pass", "slim_attn_decode", "slim_attn_decode_split",
-    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
+    "slim_attn_decode_merge", "slim_attn_decode_static", "slim_static_status", "slim_static_reset",
+    "slim_static_selftest_timeout", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -82,6 +83,9 @@ def lib():
         L.slim_attn_decode_merge.restype = ctypes.c_int
         L.slim_attn_decode_static.argtypes = [CP, P, P, P, I, I, I, F, P]
         L.slim_attn_decode_static.restype = ctypes.c_int
+        for name in ("slim_static_status", "slim_static_reset", "slim_static_selftest_timeout"):
+            getattr(L, name).argtypes = [P]
+            getattr(L, name).restype = ctypes.c_int
         L.slim_decode_step.argtypes = [CP, P, P, P, P, P, I, I, I, F, P, Z, P]
         L.slim_decode_step.restype = ctypes.c_int
         L.slim_decode_step_host.argtypes = [CP, P, P, P, P, P, Z, P, I, I, I, F, P, Z, P]
@@ -206,6 +210,21 @@ def slim_attn_decode_static(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, stre
     rc = lib().slim_attn_decode_static(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(kv_len), B, max_kv, Hq,
                                        sm_scale, _stream(stream))
     _check(rc, "slim_attn_decode_static")
+
+
+def slim_static_status(stream=None):
+    """slim_read_status for the built-in array of slim_attn_decode_static."""
+    return lib().slim_static_status(_stream(stream))
+
+
+def slim_static_reset(stream=None):
+    """Clears the built-in array's header (needed after a SLIM_ERR_TIMEOUT); allocates nothing."""
+    _check(lib().slim_static_reset(_stream(stream)), "slim_static_reset")
+
+
+def slim_static_selftest_timeout(stream=None):
+    """slim_selftest_timeout aimed at the built-in array's status word."""
+    _check(lib().slim_static_selftest_timeout(_stream(stream)), "slim_static_selftest_timeout")
 
 
 def slim_decode_step(cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None):

@@ -5,6 +5,9 @@
 // into 256-token chunks; the split pass (slim_decode_stream.cu) turns each chunk into a partial result
 // (m, l, O[128]) per query head, in SlimAttention order inside the chunk (Section 2.1: all scores, one
 // softmax, then .V); the merge pass below combines a row's partials by the log-sum-exp identity.
+#include <algorithm>
+#include <mutex>
+
 #include "slim_common.cuh"
 #include "slim_decode_params.cuh"
 
@@ -12,6 +15,14 @@ namespace slim {
 
 constexpr int kChunkTok = 256;   // tokens per partial result (two pages)
 static_assert(kDecodeHeaderBytes == SLIM_WORKSPACE_HEADER_BYTES, "the header size promised in slim.h");
+
+// Partials of a row of `len` cached tokens (never more than cap_tokens): one per 256-token chunk of the
+// tokens before the last one, then the last token's own.
+__device__ __forceinline__ int merge_row_partials(int len, int cap_tokens)
+{
+    const int L = min(max(len, 0), cap_tokens);
+    return (L == 0) ? 0 : (L - 1 + kChunkTok - 1) / kChunkTok + 1;
+}
 
 // Second pass: log-sum-exp merge of a row's chunk partials,
 //   M = max m_c;  l = sum l_c 2^(m_c - M);  o = sum O_c 2^(m_c - M) / l.
@@ -23,7 +34,7 @@ template <int kMergeGroups>
 __global__ void __launch_bounds__(kMergeGroups * kHeadDim)
 slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                          const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
-                         int B, int Hq, int n_chunks, int chunk_tokens)
+                         int B, int Hq, int n_slots, int cap_tokens)
 {
     constexpr int kMergeThreads = kMergeGroups * kHeadDim;
     __shared__ float w_s[kHeadDim];
@@ -34,9 +45,9 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
     pdl_wait();   // the split pass before this kernel must have finished writing the partials
     const int b = row / Hq;
     const int len = kv_len[b];
-    const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
-    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_chunks;
-    const float *po = part_o + (size_t)row * n_chunks * kHeadDim;
+    const int nc = merge_row_partials(len, cap_tokens);
+    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_slots;
+    const float *po = part_o + (size_t)row * n_slots * kHeadDim;
     // ---- the row's maximum
     float M = -INFINITY;
     for (int c = tid; c < nc; c += kMergeThreads) M = fmaxf(M, ml[c].x);
@@ -105,16 +116,16 @@ constexpr int kMergeWarpsPerBlock = 8;
 __global__ void __launch_bounds__(kMergeWarpsPerBlock * 32)
 slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                               const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
-                              int B, int Hq, int n_chunks, int chunk_tokens)
+                              int B, int Hq, int n_slots, int cap_tokens)
 {
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * kMergeWarpsPerBlock + (threadIdx.x >> 5);   // b * Hq + h
     pdl_wait();   // the split pass before this kernel must have finished writing the partials
     if (row >= B * Hq) return;
     const int len = __ldg(kv_len + row / Hq);
-    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_chunks;
-    const float4 *po = reinterpret_cast<const float4 *>(part_o + (size_t)row * n_chunks * kHeadDim) + lane;
-    const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
+    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_slots;
+    const float4 *po = reinterpret_cast<const float4 *>(part_o + (size_t)row * n_slots * kHeadDim) + lane;
+    const int nc = merge_row_partials(len, cap_tokens);
     float4 o[kMergeWarpBatch];
 #pragma unroll
     for (int u = 0; u < kMergeWarpBatch; ++u)
@@ -157,7 +168,7 @@ template <int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                                const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
-                               int B, int Hq, int n_chunks, int chunk_tokens)
+                               int B, int Hq, int n_slots, int cap_tokens)
 {
     __shared__ float4 acc_s[kWarps][32];
     __shared__ float m_s[kWarps], l_s[kWarps];
@@ -166,14 +177,14 @@ slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__
     pdl_wait();   // the split pass before this kernel must have finished writing the partials
     const int len = __ldg(kv_len + row / Hq);
     const int c_base = w * kMergeWarpBatch;
-    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_chunks;
-    const float4 *po = reinterpret_cast<const float4 *>(part_o + (size_t)row * n_chunks * kHeadDim) + lane;
+    const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + (size_t)row * n_slots;
+    const float4 *po = reinterpret_cast<const float4 *>(part_o + (size_t)row * n_slots * kHeadDim) + lane;
     float4 o[kMergeWarpBatch];
 #pragma unroll
     for (int u = 0; u < kMergeWarpBatch; ++u)
-        o[u] = ld_cg_now(po + (size_t)min(c_base + u, n_chunks - 1) * (kHeadDim / 4));   // n_chunks >= 32 here; slots past nc are not used
-    float2 v = (lane < kMergeWarpBatch && c_base + lane < n_chunks) ? __ldcg(ml + c_base + lane) : make_float2(-INFINITY, 0.f);
-    const int nc = min(n_chunks, (max(len, 0) + chunk_tokens - 1) / chunk_tokens);
+        o[u] = ld_cg_now(po + (size_t)min(c_base + u, n_slots - 1) * (kHeadDim / 4));   // n_slots >= 32 here; slots past nc are not used
+    float2 v = (lane < kMergeWarpBatch && c_base + lane < n_slots) ? __ldcg(ml + c_base + lane) : make_float2(-INFINITY, 0.f);
+    const int nc = merge_row_partials(len, cap_tokens);
     const bool mine = lane < kMergeWarpBatch && c_base + lane < nc;
     if (!mine) v = make_float2(-INFINITY, 0.f);
     const float Mw = warp_max(v.x);
@@ -225,8 +236,8 @@ slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv)
 {
     (void)Hkv;
-    const size_t nc = (size_t)(max_kv + kChunkTok - 1) / kChunkTok;
-    return kDecodeHeaderBytes + (size_t)B * Hq * nc * (kHeadDim + 2) * sizeof(float);
+    const size_t slots = (size_t)(max_kv + kChunkTok - 1) / kChunkTok + 1;   // a row's chunks and its last token
+    return kDecodeHeaderBytes + (size_t)B * Hq * slots * (kHeadDim + 2) * sizeof(float);
 }
 
 static DecodeParams make_params(const slim_cache_t *c, const void *q, const int32_t *kv_len, int B, int max_kv,
@@ -246,10 +257,11 @@ static DecodeParams make_params(const slim_cache_t *c, const void *q, const int3
     p.max_pages_per_seq = c->max_pages_per_seq;
     p.num_pages = c->num_pages;
     p.n_chunks = (max_kv + C - 1) / C;
+    p.n_slots = p.n_chunks + 1;
     p.scale_log2e = sm_scale * kLog2e;
     p.status = static_cast<int *>(workspace);
     p.part_o = reinterpret_cast<float *>(static_cast<char *>(workspace) + kDecodeHeaderBytes);
-    p.part_ml = p.part_o + (size_t)B * Hq * p.n_chunks * kHeadDim;
+    p.part_ml = p.part_o + (size_t)B * Hq * p.n_slots * kHeadDim;
     p.k_new = p.v_new = nullptr;
     p.out = nullptr;
     p.counters = nullptr;
@@ -283,7 +295,7 @@ int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const
     if (p.n_chunks == 0) return launch_decode_merge(c, out, kv_len, B, max_kv, Hq, workspace, stream);   // rows of zeros
     p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
     p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
-    const bool in_kernel = (long long)B * p.Hkv <= kDecodeCounterRows && p.G * p.n_chunks <= kInKernelMergeMaxPartials;
+    const bool in_kernel = (long long)B * p.Hkv <= kDecodeCounterRows && p.G * p.n_slots <= kInKernelMergeMaxPartials;
     if (in_kernel) {
         p.out = static_cast<__nv_bfloat16 *>(out);
         p.counters = reinterpret_cast<int *>(static_cast<char *>(workspace) + kDecodeStatusBytes);
@@ -299,23 +311,22 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
     int C;
     const DecodeParams p = make_params(c, nullptr, kv_len, B, max_kv, Hq, 1.f, const_cast<void *>(workspace), C);
     const int rows = B * Hq;
-    if (p.n_chunks >= 32 && p.n_chunks <= 16 * kMergeWarpBatch) {
-        const float *po = p.part_o, *pm = p.part_ml;
-        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(out);
-        if (p.n_chunks <= 4 * kMergeWarpBatch)
-            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<4>, dim3(rows), dim3(128), 0, stream, po, pm, kv_len, o, B, Hq, p.n_chunks, C));
-        else if (p.n_chunks <= 8 * kMergeWarpBatch)
-            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<8>, dim3(rows), dim3(256), 0, stream, po, pm, kv_len, o, B, Hq, p.n_chunks, C));
+    const int cap = (int)std::min<long long>((long long)c->max_pages_per_seq * kPageTokens, (long long)p.n_chunks * C);
+    const float *po = p.part_o, *pm = p.part_ml;
+    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(out);
+    if (p.n_slots >= 32 && p.n_slots <= 16 * kMergeWarpBatch) {
+        if (p.n_slots <= 4 * kMergeWarpBatch)
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<4>, dim3(rows), dim3(128), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
+        else if (p.n_slots <= 8 * kMergeWarpBatch)
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<8>, dim3(rows), dim3(256), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
         else
-            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<16>, dim3(rows), dim3(512), 0, stream, po, pm, kv_len, o, B, Hq, p.n_chunks, C));
-    } else if (p.n_chunks >= 32) {
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, (const float *)p.part_o,
-                                 (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq, p.n_chunks, C));
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<16>, dim3(rows), dim3(512), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
+    } else if (p.n_slots >= 32) {
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
     } else {
         const int blocks = (rows + kMergeWarpsPerBlock - 1) / kMergeWarpsPerBlock;
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_warp_kernel, dim3(blocks), dim3(kMergeWarpsPerBlock * 32), 0, stream,
-                                 (const float *)p.part_o, (const float *)p.part_ml, kv_len, static_cast<__nv_bfloat16 *>(out), B, Hq,
-                                 p.n_chunks, C));
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_warp_kernel, dim3(blocks), dim3(kMergeWarpsPerBlock * 32), 0, stream, po, pm, kv_len, o, B, Hq,
+                                 p.n_slots, cap));
     }
     return SLIM_OK;
 }
@@ -331,6 +342,7 @@ static __device__ __align__(256) unsigned char g_static_decode_scratch[SLIM_STAT
 
 namespace {
 constexpr int kMaxDevices = 64;
+std::mutex g_static_scratch_mu;               // guards the two tables below (host threads may make their first call together)
 void *g_static_scratch_ptr[kMaxDevices];      // device address of the array, per device ordinal
 bool g_static_scratch_ready[kMaxDevices];
 }  // namespace
@@ -342,6 +354,7 @@ static int static_scratch_address(void **ptr)
     int dev = -1;
     SLIM_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return SLIM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mu);
     if (!g_static_scratch_ready[dev]) {
         void *addr = nullptr;
         SLIM_CUDA_TRY(cudaGetSymbolAddress(&addr, g_static_decode_scratch));
@@ -378,3 +391,32 @@ int slim_attn_decode_static(const slim_cache_t *cache, const void *q, void *out,
     return launch_decode(cache, q, nullptr, nullptr, out, kv_len, B, max_kv, Hq, sm_scale, scratch, (cudaStream_t)stream);
 }
 
+// The built-in array's header (status word and merge counters) is out of the caller's reach, so these three calls
+// stand in for slim_read_status, a cudaMemset of the header and slim_selftest_timeout on an ordinary workspace.
+extern "C" __attribute__((visibility("default")))
+int slim_static_status(void *stream)
+{
+    void *scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != SLIM_OK) return rc;
+    return slim_read_status(scratch, stream);
+}
+
+extern "C" __attribute__((visibility("default")))
+int slim_static_reset(void *stream)
+{
+    void *scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != SLIM_OK) return rc;
+    SLIM_CUDA_TRY(cudaMemsetAsync(scratch, 0, SLIM_WORKSPACE_HEADER_BYTES, (cudaStream_t)stream));
+    return SLIM_OK;
+}
+
+extern "C" __attribute__((visibility("default")))
+int slim_static_selftest_timeout(void *stream)
+{
+    void *scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != SLIM_OK) return rc;
+    return slim_selftest_timeout(scratch, stream);
+}

@@ -18,16 +18,23 @@
 //    completion to the group's mbarrier and to the stages' "empty" mbarriers.
 //  * Three consumer groups of four warps (two when a kv head serves more than eight query heads) take
 //    chunks in turn.  For its chunk a group
-//      - builds the query operand: a 14-bit fixed-point copy of the G = Hq/Hkv query rows of the kv
-//        head, two signed bytes per value (columns [high bytes | low bytes]);
+//      - builds the query operand: a 22-bit fixed-point copy of the G = Hq/Hkv query rows of the kv
+//        head, three signed bytes per value (columns [high | middle | low bytes]), so that a row with a
+//        few channels hundreds of times larger than the rest keeps the small channels' precision;
 //      - S^T[token][head] = K_codes . Q^T by tcgen05.mma kind::i8: the INT8 codes are the operand as
 //        they are (the hybrid-dtype step of Section 2.2 happens inside the tensor core);
 //      - one softmax over the chunk's 256 scores per head (Section 2.1 order: all scores, softmax,
 //        then .V), thread = token, after a tensor-memory load;
 //      - O^T[dim][head] = V_codes^T . P^T, again kind::i8, V read MN-major straight from its
 //        token-major rows, P as 16-bit fixed point in two unsigned bytes;
-//      - recombines 256 * high + low exactly in int32 and writes the partial.
+//      - recombines the byte planes and writes the partial.
 //    While one group computes, the other groups' chunks and the next chunks are in flight.
+//  * The chunks cover every token of a sequence but the last one.  The last token is attended from registers by
+//    one consumer warp while the first tiles are on their way: its K and V rows come either from the caller
+//    (one-call step: the warp quantises them and stores them in the cache) or from the cache, and the warp
+//    writes the token's own partial (m, l, O) into the slot after the row's last chunk.  A decode step whose
+//    new token starts a chunk of its own therefore costs no chunk, and nothing in the kernel reads a cache row
+//    that the kernel itself wrote.
 //
 // The V scale is folded into the softmax weight (s'_j = s_j + log2 sv_j, P_j = 2^(s'_j - max s'),
 // o = sum P_j c_j / sum P_j / sv_j), so P <= 1 is normalised by the chunk's largest contribution.
@@ -47,20 +54,22 @@ constexpr int kStTile = 128;                                    // tokens per MM
 constexpr int kStChunk = 2 * kStTile;                           // tokens per chunk / partial
 constexpr int kStTailBox = 16;                                  // rows per TMA box of a ragged tile
 constexpr uint32_t kStTileBytes = kStTile * kHeadDim;           // 16 KB
-constexpr float kStQFix = 8192.f;      // |q / pow2| < 2  ->  |v| < 16384, high byte in [-64, 64]
+constexpr float kStQFix = 1048576.f;   // 2^20: |q / pow2| < 2  ->  |v| < 2^21: bytes [hi in [-32, 32] | mid | lo]
 constexpr float kStPFix = 65535.f;
 
 static_assert(kStChunk == 256, "partials are indexed by 256-token chunks (decode_workspace_bytes, merge kernel)");
 
 template <int NH, bool kAppend = false>
 struct StSmem {
-    static constexpr int N = 2 * NH;                        // MMA columns: [hi bytes of NH heads | lo bytes]
+    static constexpr int NS = (3 * NH + 15) / 16 * 16;      // score MMA columns: [hi | mid | lo bytes of NH heads], padded to 16
+    static constexpr int NP = 2 * NH;                       // output MMA columns: [hi | lo bytes of P for NH heads]
     static constexpr int kGroups = (NH <= 8) ? 3 : 2;       // consumer groups (chunks in process at a time)
     static constexpr int kThreads = kGroups * kStGroupThreads + 64 + kGroups * 32;   // groups + two producer warps + one MMA-issue warp per group
     static constexpr int kProducerWarp = kGroups * 4;
     static constexpr int kInfoSlots = 2 * kGroups;          // chunk records in flight
     static constexpr uint32_t kTmemCols = (kGroups <= 2) ? 256 : 512;   // 128 per group: S of two tiles + O
-    static constexpr int kStages = 10;                      // tile stages of the ring
+    static_assert(2 * NS + NP <= 128, "a group's accumulators fit its 128 tensor-memory columns");
+    static constexpr int kStages = (NH <= 8) ? 10 : 9;      // tile stages of the ring
     // chunk record: both scale vectors, the kv head's query rows, the chunk's coordinates
     static constexpr uint32_t kScales = 0;                  // per tile: 128 K scales, then 128 V scales
     static constexpr uint32_t kQraw = 2048;                 // bf16 [G][128]
@@ -69,10 +78,10 @@ struct StSmem {
     static constexpr uint32_t kInfo0 = kStages * kStTileBytes;
     // per consumer group
     static constexpr uint32_t kGroup0 = kInfo0 + kInfoSlots * kInfoBytes;
-    static constexpr uint32_t kPTileBytes = N * 128;        // a P^T tile, core-matrix layout
+    static constexpr uint32_t kPTileBytes = NP * 128;       // a P^T tile, core-matrix layout
     static constexpr uint32_t kP = 0;                       // two P^T tiles
-    static constexpr uint32_t kQop = 2 * kPTileBytes;       // query operand: N rows x 128 bytes, core-matrix layout
-    static constexpr uint32_t kLsum = kQop + N * 128;       // floats [NH][128]: every token thread's share of the softmax denominators
+    static constexpr uint32_t kQop = 2 * kPTileBytes;       // query operand: NS rows x 128 bytes, core-matrix layout
+    static constexpr uint32_t kLsum = kQop + NS * 128;      // floats [NH][128]: every token thread's share of the softmax denominators
     static constexpr uint32_t kRed = kLsum + NH * 512;      // floats: [NH][4] warp maxima, [NH] row scales
     static constexpr uint32_t kGroupBytes = (kRed + 5 * NH * 4 + 127) / 128 * 128;
     // block-wide: mbarriers full[kStages], empty[kStages], info full[4], info empty[4],
@@ -82,9 +91,12 @@ struct StSmem {
     static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
     static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[5]: chunks of this block, first sequence / head / chunk, that sequence's chunks
     static constexpr uint32_t kFail = kRange + 32;
-    static constexpr uint32_t kAppended = kFail + 4;       // int: consumer warps that have written their share of the new-token rows
-    static constexpr uint32_t kBytes = kFail + 8;
+    // the block table, when all of it fits: page ids are then looked up without a round trip to global memory
+    static constexpr uint32_t kTable = kFail + 16;
+    static constexpr int kTableInts = (232448 - (int)kTable) / 4;
+    static constexpr uint32_t kBytes = kTable + kTableInts * 4;
     static_assert(kRange % 16 == 0, "range record is read as int4-aligned ints");
+    static_assert(kTableInts >= 1024, "room for the block table of the configured workloads");
     static_assert(kBytes <= 232448, "shared memory budget of one block");
 };
 
@@ -126,8 +138,14 @@ __device__ __forceinline__ int st_clamped_len(const DecodeParams &p, int b)
     return min(max(__ldg(p.kv_len + b), 0), cap);
 }
 
+// The tokens of a sequence that the chunks cover: all but the last one, which is attended from registers.
+__device__ __forceinline__ int st_chunk_len(const DecodeParams &p, int b)
+{
+    return max(st_clamped_len(p, b) - 1, 0);
+}
+
 // Steps (sequence, kv head, chunk) to the next chunk in the order the work is cut in; sequences without
-// tokens are skipped.  Only called while another chunk exists, so a sequence with tokens is always found.
+// chunks are skipped.  Only called while another chunk exists, so a sequence with chunks is always found.
 __device__ __forceinline__ void st_next_chunk(const DecodeParams &p, int B, int &b, int &head, int &chunk, int &len, int &nc)
 {
     if (++chunk == nc) {
@@ -136,23 +154,96 @@ __device__ __forceinline__ void st_next_chunk(const DecodeParams &p, int B, int 
             head = 0;
             do {
                 ++b;
-                len = (b < B) ? st_clamped_len(p, b) : kStChunk;   // b < B always holds inside a block's range
+                len = (b < B) ? st_chunk_len(p, b) : kStChunk;   // b < B always holds inside a block's range
                 nc = (len + kStChunk - 1) / kStChunk;
             } while (nc == 0);
         }
     }
 }
 
-// Bounded wait until a counter in shared memory (written by another warp of the block) reaches `target`.
-__device__ __noinline__ bool st_wait_count(const volatile int *counter, int target, uint32_t max_tries)
+// floor(a / b) for 0 <= a, 0 < b: the 64-bit division is only taken when the dividend needs it
+__device__ __forceinline__ long long st_div(long long a, int b)
 {
-    while (*counter < target)
-        if (--max_tries == 0u) return false;
-    __threadfence_block();
-    return true;
+    if (((unsigned long long)a >> 32) == 0ull) return (long long)((unsigned)a / (unsigned)b);
+    return a / b;
 }
 
-// Log-sum-exp merge of the nc chunk partials of the G query heads of (sequence b, kv head `head`) by one warp:
+// The last token of (sequence b, kv head `head`), at position L - 1, attended by one warp from registers
+// (lanes 0-15 hold its K row, lanes 16-31 its V row, eight dims per lane).  With kAppend and a length that was
+// not clamped the rows are the caller's new token: they are quantised here and stored in the cache (Section
+// 2.2; exactly the codes and scales slim_kv_append writes); otherwise they are read from the cache.  For each
+// of the G query heads the token's partial - score s' = s + log2(sv), weight P = 1, so m = s', l = 1 / sv and
+// O = the V codes - goes to slot `slot` of the row; with to_out (a sequence of one token in a launch that merges
+// its own partials) the result code * sv is written straight to the output instead.
+template <bool kAppend>
+__device__ __forceinline__ void st_last_token(const DecodeParams &p, int b, int head, int L, int slot, int lane, bool to_out)
+{
+    const int kv = lane >> 4, l = lane & 15;
+    const int pos = L - 1;
+    const int page_raw = __ldg(p.block_table + (size_t)b * p.max_pages_per_seq + (pos >> 7));
+    const bool page_ok = page_raw >= 0 && page_raw < p.num_pages;
+    const int page = page_ok ? page_raw : 0;
+    const int row_in_page = pos & (kPageTokens - 1);
+    const size_t code_off = code_block_offset(page, head, kv, p.Hkv) + (size_t)row_in_page * kHeadDim;
+    const size_t scale_off = scale_block_offset(page, head, kv, p.Hkv) + row_in_page;
+    uint2 pk;
+    float scale;
+    if (kAppend && __ldg(p.kv_len + b) == L) {   // (the same for every lane of the warp)
+        const __nv_bfloat16 *src = (kv ? p.v_new : p.k_new) + ((size_t)b * p.Hkv + head) * kHeadDim;
+        pk = quantize_row16(__ldg(reinterpret_cast<const uint4 *>(src) + l), scale);
+        if (page_ok) {
+            reinterpret_cast<uint2 *>(const_cast<int8_t *>(p.codes) + code_off)[l] = pk;
+            if (l == 0) const_cast<float *>(p.scales)[scale_off] = scale;
+        }
+    } else {
+        pk = __ldg(reinterpret_cast<const uint2 *>(p.codes + code_off) + l);
+        scale = __ldg(p.scales + scale_off);
+    }
+    const float sk = __shfl_sync(0xffffffffu, scale, 0);
+    const float sv = fmaxf(__shfl_sync(0xffffffffu, scale, 16), kMinScale);
+    float c[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        c[i] = (float)(int)(int8_t)((pk.x >> (8 * i)) & 0xFFu);
+        c[4 + i] = (float)(int)(int8_t)((pk.y >> (8 * i)) & 0xFFu);
+    }
+    const float lsv = __log2f(sv), rsv = st_rcp(sv), ks = sk * p.scale_log2e;
+    for (int h = 0; h < p.G; ++h) {
+        const size_t row = (size_t)b * p.Hq + (size_t)head * p.G + h;
+        if (to_out) {
+            if (kv == 1) {
+                uint32_t w[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    __nv_bfloat162 x = __floats2bfloat162_rn(c[2 * i] * sv, c[2 * i + 1] * sv);
+                    w[i] = *reinterpret_cast<uint32_t *>(&x);
+                }
+                reinterpret_cast<uint4 *>(p.out + row * kHeadDim)[l] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            continue;
+        }
+        const uint4 qv = __ldg(reinterpret_cast<const uint4 *>(p.q + row * kHeadDim) + l);
+        const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
+        float dot = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            dot = fmaf(bf16_bits_to_float(qw[i] & 0xFFFFu), c[2 * i], dot);
+            dot = fmaf(bf16_bits_to_float(qw[i] >> 16), c[2 * i + 1], dot);
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // lanes 0-15: q . k codes
+        const float s = __shfl_sync(0xffffffffu, dot, 0);
+        const size_t ps = row * p.n_slots + slot;
+        if (kv == 1) {
+            float4 *dst = reinterpret_cast<float4 *>(p.part_o + ps * kHeadDim + 8 * l);
+            dst[0] = make_float4(c[0], c[1], c[2], c[3]);
+            dst[1] = make_float4(c[4], c[5], c[6], c[7]);
+        }
+        if (lane == 0) *reinterpret_cast<float2 *>(p.part_ml + ps * 2) = make_float2(fmaf(s, ks, lsv), rsv);
+    }
+}
+
+// Log-sum-exp merge of the nc partials (the chunks' and the last token's) of the G query heads of (sequence b, kv head `head`) by one warp:
 //   M = max m_c;  l = sum l_c 2^(m_c - M);  o = sum O_c 2^(m_c - M) / l   (a lane owns four head dims).
 // The caller has made sure that every partial of the pair is visible; they are read past the L1 cache.
 __device__ __forceinline__ void st_merge_rows(const DecodeParams &p, int b, int head, int nc, int lane)
@@ -160,8 +251,8 @@ __device__ __forceinline__ void st_merge_rows(const DecodeParams &p, int b, int 
     constexpr int kBatch = 12;   // partial outputs requested before the first of them is used
     for (int h = 0; h < p.G; ++h) {
         const size_t row = (size_t)b * p.Hq + (size_t)head * p.G + h;
-        const float2 *ml = reinterpret_cast<const float2 *>(p.part_ml) + row * p.n_chunks;
-        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + row * p.n_chunks * kHeadDim) + lane;
+        const float2 *ml = reinterpret_cast<const float2 *>(p.part_ml) + row * p.n_slots;
+        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + row * p.n_slots * kHeadDim) + lane;
         // every load of the first round is in flight before anything waits for one of them
         float4 o[kBatch];
 #pragma unroll
@@ -211,7 +302,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                           const DecodeParams p, const int B)
 {
     using L = StSmem<NH, kAppend>;
-    constexpr int N = L::N;
+    constexpr int NS = L::NS, NP = L::NP;
     constexpr int S = L::kStages;
     constexpr int kStGroups = L::kGroups, kStInfoSlots = L::kInfoSlots;
     constexpr int kPW = L::kProducerWarp;
@@ -230,7 +321,9 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kTmemSlot);
     int *range = reinterpret_cast<int *>(smem + L::kRange);
     volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
-    volatile int *appended = reinterpret_cast<volatile int *>(smem + L::kAppended);
+    int *table = reinterpret_cast<int *>(smem + L::kTable);
+    const bool use_table = (long long)B * p.max_pages_per_seq <= (long long)L::kTableInts;
+    const int table_ints = use_table ? B * p.max_pages_per_seq : 0;
 
     pdl_launch_dependents();   // the merge kernel queued behind this one may be scheduled; it waits for our completion
     if (tid == 0) {
@@ -251,7 +344,6 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         }
         tc::mbar_init_fence();
         *fail = 0;
-        *appended = 0;
     }
     if (warp == kPW) {
         tc::tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
@@ -260,10 +352,10 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         pdl_wait();
         // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order.  The work is cut
         //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.
-        const int len_first = (lane < B) ? st_clamped_len(p, lane) : 0;   // the first 32 sequences stay in registers
-        auto seq_len = [&](int base) {
+        const int len_first = (lane < B) ? st_chunk_len(p, lane) : 0;   // the first 32 sequences stay in registers
+        auto seq_len = [&](int base) {   // tokens of sequence base + lane that the chunks cover
             const int b = base + lane;
-            return (base == 0) ? len_first : ((b < B) ? st_clamped_len(p, b) : 0);
+            return (base == 0) ? len_first : ((b < B) ? st_chunk_len(p, b) : 0);
         };
         long long tiles_all = 0;
         for (int base = 0; base < B; base += 32)
@@ -287,8 +379,8 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const int nt_l = __shfl_sync(0xffffffffu, nt, l), nc_l = __shfl_sync(0xffffffffu, nc, l);
                     const long long tb = tiles_pre + __shfl_sync(0xffffffffu, it, l) - nt_l;
                     const long long cb = chunks_pre + __shfl_sync(0xffffffffu, ic, l) - nc_l;
-                    const long long r = x - tb * p.Hkv;              // < Hkv * nt_l
-                    const int head = (int)(r / nt_l), d = (int)(r % nt_l);
+                    const int r = (int)(x - tb * p.Hkv);             // < Hkv * nt_l
+                    const int head = r / nt_l, d = r - head * nt_l;
                     return cb * p.Hkv + (long long)head * nc_l + min(nc_l, (d + 1) / 2);
                 }
                 tiles_pre += __shfl_sync(0xffffffffu, it, 31);
@@ -296,8 +388,8 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             }
             return chunks_pre * p.Hkv;
         };
-        const long long i0 = chunks_before(total_tiles * blockIdx.x / gridDim.x);
-        const long long i1 = chunks_before(total_tiles * (blockIdx.x + 1) / gridDim.x);
+        const long long i0 = chunks_before(st_div(total_tiles * blockIdx.x, (int)gridDim.x));
+        const long long i1 = chunks_before(st_div(total_tiles * (blockIdx.x + 1), (int)gridDim.x));
         int b0 = 0, head0 = 0, chunk0 = 0, nc0 = 1;
         if (i1 > i0) {
             long long prefix = 0;   // chunks of the sequences before `base`
@@ -314,10 +406,10 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const int l = __ffs(hit) - 1;
                     const int nc_l = __shfl_sync(0xffffffffu, nc, l);
                     const long long before = prefix + __shfl_sync(0xffffffffu, incl, l) - nc_l;
-                    const long long r = i0 - before * p.Hkv;   // < Hkv * nc_l
+                    const int r = (int)(i0 - before * p.Hkv);   // < Hkv * nc_l
                     b0 = base + l;
-                    head0 = (int)(r / nc_l);
-                    chunk0 = (int)(r % nc_l);
+                    head0 = r / nc_l;
+                    chunk0 = r - head0 * nc_l;
                     nc0 = nc_l;
                     break;
                 }
@@ -335,7 +427,12 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         // rows of the query operand that belong to no head stay zero for the whole launch
         const int g = warp >> 2, gtid = tid & 127;
         unsigned char *qop = smem + L::kGroup0 + g * L::kGroupBytes + L::kQop;
-        for (int i = gtid * 16; i < N * 128; i += kStGroupThreads * 16) *reinterpret_cast<uint4 *>(qop + i) = make_uint4(0, 0, 0, 0);
+        for (int i = gtid * 16; i < NS * 128; i += kStGroupThreads * 16) *reinterpret_cast<uint4 *>(qop + i) = make_uint4(0, 0, 0, 0);
+    } else if (use_table) {
+        // the second producer warp and the MMA-issue warps copy the block table while the lengths are on their way
+        pdl_wait();
+        constexpr int kCopyThreads = L::kThreads - (kPW + 1) * 32;
+        for (int i = tid - (kPW + 1) * 32; i < table_ints; i += kCopyThreads) table[i] = __ldg(p.block_table + i);
     }
     tc::fence_proxy_async();
     tc::fence_before_sync();
@@ -361,21 +458,25 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         if (lane == 0 && cnt > 0) {
             pdl_wait();   // (returns at once: the earlier kernel was already waited for before the lengths were read)
             int b = range[1], head = range[2], chunk = range[3];
-            int len = st_clamped_len(p, b);
+            int len = st_chunk_len(p, b);
             int nc = (len + kStChunk - 1) / kStChunk;
             auto page_ids = [&](int bb, int cc) {
-                const int32_t *bt = p.block_table + (size_t)bb * p.max_pages_per_seq + cc * 2;
                 int2 r;
-                r.x = (cc * 2 < p.max_pages_per_seq) ? __ldg(bt) : 0;
-                r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
+                if (use_table) {
+                    const int at = bb * p.max_pages_per_seq + cc * 2;
+                    r.x = (cc * 2 < p.max_pages_per_seq) ? table[at] : 0;
+                    r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? table[at + 1] : 0;
+                } else {
+                    const int32_t *bt = p.block_table + (size_t)bb * p.max_pages_per_seq + cc * 2;
+                    r.x = (cc * 2 < p.max_pages_per_seq) ? __ldg(bt) : 0;
+                    r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
+                }
                 return r;
             };
+            const uint64_t stream_policy = tc::policy_evict_first();   // cache rows are read once per launch
             int2 pg = page_ids(b, chunk);
             int stage = 0;
             uint32_t stage_ph = 0;   // parity of the stage's current use
-            // one-call step: list index of the block's first chunk that holds a new token's slot (the last chunk of
-            // the first sequence and head); the consumer warps must have written the block's new rows before it is fetched
-            const int n_first_new = kAppend ? range[4] - 1 - range[3] : -1;
             for (int n = 0; n < cnt; ++n) {
                 const int cb = b, chead = head, cchunk = chunk;
                 const int n_tok = min(kStChunk, len - chunk * kStChunk);
@@ -384,12 +485,6 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 if (n + 1 < cnt) {
                     st_next_chunk(p, B, b, head, chunk, len, nc);
                     pg = page_ids(min(b, B - 1), chunk);
-                }
-                if (kAppend && n == n_first_new) {
-                    if (!st_wait_count(appended, kPW, ok ? (1u << 20) : 1u)) {
-                        ok = false;
-                        *fail = 1;
-                    }
                 }
                 int page[2] = {cpg.x, cpg.y};
                 int rows16[2];
@@ -417,8 +512,8 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
                     for (int t = 0; t < 2; ++t)
                         if (t < n_tiles)
-                            tc::bulk_load(info_addr + L::kScales + t * 1024, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
-                                          1024u, bar_info_full(islot));
+                            tc::bulk_load_hint(info_addr + L::kScales + t * 1024, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
+                                               1024u, bar_info_full(islot), stream_policy);
                     if (need_q)
                         tc::bulk_load(info_addr + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes,
                                       bar_info_full(islot));
@@ -436,10 +531,10 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                             const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
                             const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
                             if (rows16[t] == kStTile) {
-                                tc::tma_load_2d(dst, &map_tile, 0, row0, full);
+                                tc::tma_load_2d_hint(dst, &map_tile, 0, row0, full, stream_policy);
                             } else {
                                 for (int r = 0; r < rows16[t]; r += kStTailBox)
-                                    tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
+                                    tc::tma_load_2d_hint(dst + r * kHeadDim, &map_tail, 0, row0 + r, full, stream_policy);
                             }
                             ++tiles_issued;
                             if (++stage == S) {
@@ -457,8 +552,8 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         if (lane == 0) {
             const uint32_t grp_addr = sbase + L::kGroup0 + g * L::kGroupBytes;
             const uint32_t tm = tmem + (uint32_t)g * 128u;
-            constexpr uint32_t idesc_s = tc::instr_desc(2, 1, 1, false, false, 128, N);    // s32 <- s8 (K-major) x s8 (K-major)
-            constexpr uint32_t idesc_pv = tc::instr_desc(2, 1, 0, true, false, 128, N);    // s32 <- s8 (MN-major) x u8 (K-major)
+            constexpr uint32_t idesc_s = tc::instr_desc(2, 1, 1, false, false, 128, NS);   // s32 <- s8 (K-major) x s8 (K-major)
+            constexpr uint32_t idesc_pv = tc::instr_desc(2, 1, 0, true, false, 128, NP);   // s32 <- s8 (MN-major) x u8 (K-major)
             // operand descriptors are built once; an MMA step only adds a constant to the address field
             const uint64_t dk0 = tc::smem_desc(sbase, 16, 1024, tc::kSwizzle128B);         // a K tile in stage 0
             const uint64_t dv0 = tc::smem_desc(sbase, 1024, 1024, tc::kSwizzle128B);       // a V tile in stage 0 (MN-major)
@@ -493,7 +588,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                         const uint64_t a = dk0 + (uint64_t)((uint32_t)st[t] * (kStTileBytes >> 4));
 #pragma unroll
                         for (int j = 0; j < 4; ++j)   // 32 dims per step: 32 bytes inside the swizzle span; 256 bytes of the query operand
-                            tc::mma_i8(tm + t * N, a + (uint64_t)(j * 2), dq + (uint64_t)(j * 16), idesc_s, j > 0);
+                            tc::mma_i8(tm + t * NS, a + (uint64_t)(j * 2), dq + (uint64_t)(j * 16), idesc_s, j > 0);
                     }
                 }
                 tc::commit(bar_mma_s(g));
@@ -512,7 +607,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                         const uint64_t a = dv0 + (uint64_t)((uint32_t)st[n_tiles + t] * (kStTileBytes >> 4));
 #pragma unroll
                         for (int j = 0; j < 4; ++j)   // 32 tokens per step: 4 KB down the V tile; 256 bytes of the P^T tile
-                            tc::mma_i8(tm + 2 * N, a + (uint64_t)(j * 256), dp + (uint64_t)((t * L::kPTileBytes + j * 256) >> 4), idesc_pv,
+                            tc::mma_i8(tm + 2 * NS, a + (uint64_t)(j * 256), dp + (uint64_t)((t * L::kPTileBytes + j * 256) >> 4), idesc_pv,
                                        (t > 0) || (j > 0));
                     }
                 }
@@ -534,56 +629,38 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         const int bar_id = 1 + g;
         int q_b = -1, q_head = -1;                                 // whose query rows the operand buffer holds
 
-        if (kAppend) {
-            // ---- one-call step: the block that owns the last chunk of a (sequence, kv head) quantises that pair's
-            //      new K row (lanes 0-15) and V row (lanes 16-31) into slot kv_len - 1 of the cache before its
-            //      producers fetch that chunk; every other chunk of the pair holds older tokens only.  The pairs
-            //      whose last chunk lies in this block's range are dealt to the consumer warps in turn, here, while
-            //      the first tiles are on their way.
+        {
+            // ---- the last token of every (sequence, kv head) is attended from registers, here, while the first tiles
+            //      are on their way (st_last_token).  A pair with chunks belongs to the block whose range holds its
+            //      last chunk; those pairs are dealt to the block's consumer warps in turn, from the last warp down (the
+            //      first group takes the block's first chunk).  A sequence of one token has no chunk: its pairs are
+            //      dealt to the blocks by index.
+            pdl_wait();
             if (cnt > 0) {
-                pdl_wait();
                 int b = range[1], head = range[2];
-                int len = st_clamped_len(p, b);
+                int L = st_clamped_len(p, b);
                 int nc = range[4];
                 int last = nc - 1 - range[3];   // list index of the pair's last chunk
-                const int kv = lane >> 4, l = lane & 15;
                 for (int r = 0; last < cnt; ++r) {
-                    // dealt from the last consumer warp down: the first group, which takes the block's first chunk,
-                    // gets a row only when a block owns more than eight new tokens
-                    if (kPW - 1 - r % kPW == warp) {
-                        const int pos = len - 1;
-                        // a length beyond the page table or the launch's max_kv was clamped: its token has no slot
-                        const bool has_slot = __ldg(p.kv_len + b) == len;
-                        const __nv_bfloat16 *src = (kv ? p.v_new : p.k_new) + ((size_t)b * p.Hkv + head) * kHeadDim;
-                        const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(src) + l);
-                        const int page = __ldg(p.block_table + (size_t)b * p.max_pages_per_seq + (pos >> 7));
-                        float scale;
-                        const uint2 pk = quantize_row16(raw, scale);
-                        if (has_slot && page >= 0 && page < p.num_pages) {
-                            const int slot = pos & (kPageTokens - 1);
-                            int8_t *dst = const_cast<int8_t *>(p.codes) + code_block_offset(page, head, kv, p.Hkv) + (size_t)slot * kHeadDim;
-                            reinterpret_cast<uint2 *>(dst)[l] = pk;
-                            if (l == 0) const_cast<float *>(p.scales)[scale_block_offset(page, head, kv, p.Hkv) + slot] = scale;
-                        }
-                    }
-                    // the next pair with tokens
+                    if (kPW - 1 - r % kPW == warp) st_last_token<kAppend>(p, b, head, L, nc, lane, false);
+                    // the next pair with chunks
                     if (++head == p.Hkv) {
                         head = 0;
                         do {
                             ++b;
-                            len = (b < B) ? st_clamped_len(p, b) : 0;
-                        } while (b < B && len == 0);
+                            L = (b < B) ? st_clamped_len(p, b) : 0;
+                        } while (b < B && L < 2);
                         if (b >= B) break;
-                        nc = (len + kStChunk - 1) / kStChunk;
+                        nc = (L - 1 + kStChunk - 1) / kStChunk;
                     }
                     last += nc;
                 }
             }
-            // the rows are at device scope and ordered before copies of the async proxy; then the warp is counted
-            __threadfence();
-            tc::fence_proxy_async_global();
-            __syncwarp();
-            if (lane == 0) atomicAdd_block(const_cast<int *>(appended), 1);
+            const long long pairs = (long long)B * p.Hkv;
+            for (long long pr = blockIdx.x + (long long)warp * gridDim.x; pr < pairs; pr += (long long)kPW * gridDim.x) {
+                const int b = (int)st_div(pr, p.Hkv), head = (int)(pr - (long long)b * p.Hkv);
+                if (st_clamped_len(p, b) == 1) st_last_token<kAppend>(p, b, head, 1, 0, lane, kMerge);
+            }
         }
         for (int n = g; n < cnt; n += kStGroups) {
             const int islot = n % kStInfoSlots;
@@ -608,18 +685,23 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const float am = warp_max(fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
                     const float p2 = pow2_floor(am);
                     const float f = pow2_recip(p2) * kStQFix;
-                    uint32_t lo_w = 0, hi_w = 0;
+                    uint32_t lo_w = 0, mid_w = 0, hi_w = 0;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        // v = round(x * f), |v| < 16384, as the low 16 bits of 1.5 * 2^23 + v (two's complement)
-                        const int v = (int)(int16_t)(__float_as_uint(fmaf(x[i], f, 12582912.f)) & 0xFFFFu);
-                        const int hi = (v + 128) >> 8;            // v = 256 * hi + lo with lo in [-128, 127]
-                        lo_w |= ((uint32_t)v & 0xFFu) << (8 * i);
+                        // v = round(x * f), |v| < 2^21, as v = 65536 hi + 256 mid + lo with mid, lo in [-128, 127]
+                        const int v = __float2int_rn(x[i] * f);
+                        const int lo = (v << 24) >> 24;
+                        const int v1 = (v - lo) >> 8;
+                        const int mid = (v1 << 24) >> 24;
+                        const int hi = (v1 - mid) >> 8;
+                        lo_w |= ((uint32_t)lo & 0xFFu) << (8 * i);
+                        mid_w |= ((uint32_t)mid & 0xFFu) << (8 * i);
                         hi_w |= ((uint32_t)hi & 0xFFu) << (8 * i);
                     }
                     if (lane == 0) rowscale[h] = p2 * p.scale_log2e * (1.f / kStQFix);
                     *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(h, 4 * lane)) = hi_w;
-                    *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(NH + h, 4 * lane)) = lo_w;
+                    *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(NH + h, 4 * lane)) = mid_w;
+                    *reinterpret_cast<uint32_t *>(grp + L::kQop + st_core_off(2 * NH + h, 4 * lane)) = lo_w;
                 }
             }
             // this thread's two tokens
@@ -645,7 +727,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             __syncwarp();   // reconverge after the wait loop: the tensor-memory loads below are warp-aligned
             tc::fence_after_sync();
 
-            // ---- S^T from tensor memory: row = token, columns [hi | lo] per head
+            // ---- S^T from tensor memory: row = token, columns [hi | mid | lo] per head
             float s[2][NH];
             float mloc[NH];
 #pragma unroll
@@ -653,18 +735,19 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
                 if (t < n_tiles) {
-                    uint32_t r[N];
+                    uint32_t r[NS];
 #pragma unroll
-                    for (int c16 = 0; c16 < N / 16; ++c16) {
+                    for (int c16 = 0; c16 < NS / 16; ++c16) {
                         uint32_t tmp[16];
-                        tc::tmem_ld16(tm + lane_base + t * N + c16 * 16, tmp);
+                        tc::tmem_ld16(tm + lane_base + t * NS + c16 * 16, tmp);
 #pragma unroll
                         for (int i = 0; i < 16; ++i) r[c16 * 16 + i] = tmp[i];
                     }
                     tc::tmem_ld_wait();
 #pragma unroll
                     for (int h = 0; h < NH; ++h) {
-                        const float x = (float)(((int)r[h] << 8) + (int)r[NH + h]);
+                        // 65536 hi + 256 mid + lo; each plane's sum is below 2^22 in magnitude
+                        const float x = fmaf((float)(int)r[h], 65536.f, (float)(((int)r[NH + h] << 8) + (int)r[2 * NH + h]));
                         s[t][h] = (valid[t] && h < p.G) ? fmaf(x, sk[t] * rowscale[h], lsv[t]) : -INFINITY;
                         mloc[h] = fmaxf(mloc[h], s[t][h]);
                     }
@@ -714,11 +797,11 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 
             // ---- O^T from tensor memory: row = head dim, columns [hi | lo] per head; one partial per head
             {
-                uint32_t r[N];
+                uint32_t r[NP];
 #pragma unroll
-                for (int c16 = 0; c16 < N / 16; ++c16) {
+                for (int c16 = 0; c16 < NP / 16; ++c16) {
                     uint32_t tmp[16];
-                    tc::tmem_ld16(tm + lane_base + 2 * N + c16 * 16, tmp);
+                    tc::tmem_ld16(tm + lane_base + 2 * NS + c16 * 16, tmp);
 #pragma unroll
                     for (int i = 0; i < 16; ++i) r[c16 * 16 + i] = tmp[i];
                 }
@@ -726,7 +809,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
                 for (int h = 0; h < NH; ++h) {
                     if (h < p.G) {
-                        const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_chunks + chunk;
+                        const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_slots + chunk;
                         p.part_o[ps * kHeadDim + gtid] = (float)(((int)r[h] << 8) + (int)r[NH + h]) * (1.f / kStPFix);
                     }
                 }
@@ -746,7 +829,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
 #pragma unroll
                 for (int o = kLanesPerHead / 2; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
                 if (seg == 0 && h < p.G) {
-                    const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_chunks + chunk;
+                    const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_slots + chunk;
                     const float4 mw = *reinterpret_cast<const float4 *>(red_m + h * 4);
                     p.part_ml[ps * 2] = fmaxf(fmaxf(mw.x, mw.y), fmaxf(mw.z, mw.w));
                     p.part_ml[ps * 2 + 1] = l;
@@ -772,17 +855,19 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 for (int r = 0; remaining > 0; ++r) {
                     const int mine = min(nc - first, remaining);
                     if (r % kPW == warp) {
+                        // the block that holds the pair's last chunk also wrote the last token's partial (slot nc)
+                        const int wrote = mine + ((first + mine == nc) ? 1 : 0);
                         bool complete = mine == nc;
                         if (!complete) {
                             int old = 0;
-                            if (lane == 0) old = atomicAdd(p.counters + b * p.Hkv + head, mine);
-                            complete = __shfl_sync(0xffffffffu, old, 0) + mine == nc;
+                            if (lane == 0) old = atomicAdd(p.counters + b * p.Hkv + head, wrote);
+                            complete = __shfl_sync(0xffffffffu, old, 0) + wrote == nc + 1;
                             if (complete) {
                                 if (lane == 0) p.counters[b * p.Hkv + head] = 0;   // ready for the next launch
                                 __threadfence();   // the other blocks' counts were seen: their partials are visible after this
                             }
                         }
-                        if (complete) st_merge_rows(p, b, head, nc, lane);
+                        if (complete) st_merge_rows(p, b, head, nc + 1, lane);
                     }
                     remaining -= mine;
                     first = 0;
@@ -791,13 +876,14 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                         int len;
                         do {
                             ++b;
-                            len = (b < B) ? st_clamped_len(p, b) : kStChunk;   // b < B always holds inside the range
+                            len = (b < B) ? st_chunk_len(p, b) : kStChunk;   // b < B always holds inside the range
                         } while (len == 0);
                         nc = (len + kStChunk - 1) / kStChunk;
                     }
                 }
             }
-            // sequences without tokens have no chunk and therefore no merge: their rows are zero
+            // sequences without tokens have no partial and therefore no merge: their rows are zero (a sequence of one
+            // token was written by the warp that attended it)
             for (int b = blockIdx.x; b < B; b += gridDim.x) {
                 if (st_clamped_len(p, b) != 0) continue;
                 uint4 *dst = reinterpret_cast<uint4 *>(p.out + (size_t)b * p.Hq * kHeadDim);

@@ -66,9 +66,6 @@ __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fenc
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
 // Makes generic-proxy writes to shared memory (st.shared, cp.async) visible to the tensor-core (async) proxy.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-// The same for global memory: orders this thread's earlier ordinary stores to global memory before later
-// reads of them by the copy engine (TMA / bulk copies issued after a synchronisation with this thread).
-__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;\n" ::: "memory"); }
 
 // ---------------------------------------------------------------- tensor memory
 // Allocate / free `cols` (power of two >= 32) TMEM columns; executed by one whole warp.
@@ -170,7 +167,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar_smem, uint32_t parity, u
     return false;
 }
 
-// ---------------------------------------------------------------- TMA (no multicast anywhere)
+// ---------------------------------------------------------------- TMA: every copy is addressed to this block alone
 // 2-D tiled tensor copy global -> shared; x (the innermost coordinate, in elements) must keep
 // x * element size a multiple of 16 bytes.  Completion is counted in bytes on the mbarrier.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void *tmap, int x, int y, uint32_t mbar_smem)
@@ -180,12 +177,36 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void *tmap,
         "l"(tmap), "r"(x), "r"(y), "r"(mbar_smem)
         : "memory");
 }
+// The same copy with a cache policy for the L2 (see policy_evict_first).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst_smem, const void *tmap, int x, int y, uint32_t mbar_smem, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;\n" ::"r"(
+            dst_smem),
+        "l"(tmap), "r"(x), "r"(y), "r"(mbar_smem), "l"(policy)
+        : "memory");
+}
+// L2 policy for data that is read once: its lines are the first to be replaced, so that a long stream does not
+// push the small tables and partial results that are read again out of the L2.
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
+    return policy;
+}
 // Untiled bulk copy global -> shared: both addresses 16-byte aligned, size a multiple of 16.
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t mbar_smem)
 {
     asm volatile(
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst_smem),
         "l"(src), "r"(bytes), "r"(mbar_smem)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t mbar_smem, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(dst_smem),
+        "l"(src), "r"(bytes), "r"(mbar_smem), "l"(policy)
         : "memory");
 }
 // Barrier among `count` threads (a multiple of 32) of the block, id 1..15.

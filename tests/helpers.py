@@ -96,3 +96,19 @@ def mantissa_sweep_bits(exponents, offsets=range(0, 10), subnormal_amax=(1, 2, 3
         row = np.where(mant <= m, mant, mant % (m + 1)).astype(np.uint32) | sign
         rows.append(row.astype(np.uint16))
     return np.stack(rows)
+
+
+MAX_ABS = 2e-2     # output tolerance against the fp64 oracle: max-abs ...
+MEAN_ABS = 2e-3    # ... and mean-abs
+
+
+def output_bound(want_f64):
+    """Per-element bound on |bf16 output - fp64 oracle value|.
+
+    The flat 2e-2 wherever a bf16 output can meet it: below magnitude 8 the bf16 half-ulp is at most 2^-6 =
+    1.56e-2.  From magnitude 8 on the half-ulp is 2^-5 or more, so the correctly rounded oracle value itself may
+    miss 2e-2; there the bound is the bf16 half-ulp of the oracle value plus the arithmetic share that the flat
+    bound leaves in the binade below, 2e-2 - 2^-6 = 4.4e-3."""
+    a = np.abs(want_f64)
+    half_ulp = 2.0 ** (np.floor(np.log2(np.maximum(a, 1.0))) - 8)   # bf16 has 8 significant bits
+    return np.where(a >= 8.0, half_ulp + (MAX_ABS - 2.0 ** -6), MAX_ABS)

@@ -3,10 +3,12 @@
 Codes and scale bits must be identical; attention outputs (bf16) must be within
 max-abs 2e-2 and mean-abs 2e-3 of the fp64 oracle evaluated on the same codes.
 
-A bf16 number of magnitude >= 8 has a half-ulp of 2^-5 > 2e-2, so no bf16 output can
-meet a flat 2e-2 bound there (the outlier channels of workloads 2 and 4 produce such
-values).  For |o| >= 4 the bound is therefore 2e-2 plus the bf16 rounding allowance
-|o| * 2^-8; below 4 it is the flat 2e-2.
+The flat 2e-2 holds wherever a bf16 output can meet it: below magnitude 8 the bf16
+half-ulp is at most 2^-6 = 1.56e-2.  From magnitude 8 on the half-ulp is 2^-5 or more,
+so the correctly rounded oracle value itself may miss 2e-2 (the outlier channels of
+workloads 2 and 4 produce a handful of such outputs).  There the bound is the bf16
+half-ulp of the oracle value plus the arithmetic share the flat bound leaves in the
+binade below, 2e-2 - 2^-6 = 4.4e-3.
 """
 import numpy as np
 import pytest
@@ -14,12 +16,9 @@ import torch
 
 from oracle import slim_oracle as so
 from paper_2407_07304_b200 import workloads
-from helpers import bf16_bits, mantissa_sweep_bits
+from helpers import MAX_ABS, MEAN_ABS, bf16_bits, mantissa_sweep_bits, output_bound
 
 pytestmark = pytest.mark.gpu
-
-MAX_ABS = 2e-2
-MEAN_ABS = 2e-3
 
 
 def _oracle_cache(w):
@@ -42,14 +41,22 @@ def _assert_cache_bits(run, oc):
         assert np.array_equal(vs.numpy().view(np.uint32), oc[b][3][:T].view(np.uint32)), f"V scales differ (seq {b})"
 
 
+RELAXED = {"elements": 0, "worst_excess_over_flat": 0.0}   # how often the bound above magnitude 8 was needed
+
+
 def _assert_close(got_bf16, want_f64, what):
     got = got_bf16.float().cpu().numpy().astype(np.float64)
     err = np.abs(got - want_f64)
     assert np.isfinite(got).all(), f"{what}: non-finite output"
-    bound = np.where(np.abs(want_f64) >= 4.0, MAX_ABS + np.abs(want_f64) * 2.0 ** -8, MAX_ABS)
+    bound = output_bound(want_f64)
     i = np.unravel_index((err - bound).argmax(), err.shape)
-    assert (err <= bound).all(), f"{what}: abs error {err[i]:.3e} at {i}: got {got[i]!r} want {want_f64[i]!r}"
+    assert (err <= bound).all(), f"{what}: abs error {err[i]:.3e} (bound {bound[i]:.3e}) at {i}: got {got[i]!r} want {want_f64[i]!r}"
     assert err.mean() <= MEAN_ABS, f"{what}: mean-abs {err.mean():.3e}"
+    over = err > MAX_ABS
+    if over.any():
+        RELAXED["elements"] += int(over.sum())
+        RELAXED["worst_excess_over_flat"] = max(RELAXED["worst_excess_over_flat"], float((err - MAX_ABS).max()))
+        print(f"{what}: {int(over.sum())} element(s) of magnitude >= 8 above the flat bound, worst {err[over].max():.3e}")
     return err.max(), err.mean()
 
 
@@ -231,6 +238,26 @@ def test_random_shapes_against_the_oracle():
         steps = rng.choice([0, 1, 2, 3])
         one = steps > 0 and rng.random() < 0.5
         _check(_custom(B, Hkv * G, Hkv, pre, bulk, steps, rng.randint(0, 10 ** 6)), one_call_step=one)
+
+
+@pytest.mark.parametrize("factor", [8.0, 64.0, 512.0])
+@pytest.mark.parametrize("n_channels", [1, 4])
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 1)])
+def test_query_outlier_channels(factor, n_channels, Hq, Hkv):
+    # Query rows with a few channels far above the rest (as trained models have): the other channels must keep
+    # their precision.  The same channels of K are divided by the factor, so the scores stay of order one and the
+    # softmax does not saturate (a saturated softmax would hide an inaccurate score).  Prefill of 299 and 2048
+    # tokens, then decode steps at 300 / 2049 and 301 / 2050 cached tokens, and a batch of very short contexts
+    # (1..6 tokens) where two or three keys share the weight and a score error shows undiluted.
+    for lens, seed in (([299, 2048], 4100), ([1, 2, 3, 5], 4200)):
+        B = len(lens)
+        w = _custom(B, Hq, Hkv, lens, [0] * B, 2, seed + int(factor) + n_channels)
+        ch = torch.randperm(128, generator=torch.Generator().manual_seed(seed))[:n_channels]
+        for b in range(B):
+            w.q_prefill[b][:, :, ch] = (w.q_prefill[b][:, :, ch].float() * factor).to(torch.bfloat16)
+            w.k[b][:, :, ch] = (w.k[b][:, :, ch].float() / factor).to(torch.bfloat16)
+        w.q_decode[:, :, :, ch] = (w.q_decode[:, :, :, ch].float() * factor).to(torch.bfloat16)
+        _check(w)
 
 
 @pytest.mark.parametrize("length", [8200, 12345, 20000, 40001, 66000])
