@@ -89,14 +89,10 @@ struct StSmem {
     static constexpr uint32_t kBar = kGroup0 + kGroups * kGroupBytes;
     static constexpr int kNumBars = 2 * kStages + 2 * kInfoSlots + 4 * kGroups;
     static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
-    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[5]: chunks of this block, first sequence / head / chunk, that sequence's chunks
+    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[6]: chunks of this block, first sequence / head / chunk, that sequence's chunks and chunk tokens
     static constexpr uint32_t kFail = kRange + 32;
-    // the block table, when all of it fits: page ids are then looked up without a round trip to global memory
-    static constexpr uint32_t kTable = kFail + 16;
-    static constexpr int kTableInts = (232448 - (int)kTable) / 4;
-    static constexpr uint32_t kBytes = kTable + kTableInts * 4;
+    static constexpr uint32_t kBytes = kFail + 16;
     static_assert(kRange % 16 == 0, "range record is read as int4-aligned ints");
-    static_assert(kTableInts >= 1024, "room for the block table of the configured workloads");
     static_assert(kBytes <= 232448, "shared memory budget of one block");
 };
 
@@ -321,12 +317,105 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::kTmemSlot);
     int *range = reinterpret_cast<int *>(smem + L::kRange);
     volatile int *fail = reinterpret_cast<volatile int *>(smem + L::kFail);
-    int *table = reinterpret_cast<int *>(smem + L::kTable);
-    const bool use_table = (long long)B * p.max_pages_per_seq <= (long long)L::kTableInts;
-    const int table_ints = use_table ? B * p.max_pages_per_seq : 0;
 
     pdl_launch_dependents();   // the merge kernel queued behind this one may be scheduled; it waits for our completion
-    if (tid == 0) {
+
+    // ---- the producers' walk over the block's chunk list.  State of one walker (each producer thread has its own):
+    int w_b = 0, w_head = 0, w_chunk = 0, w_len = 0, w_nc = 1;   // the chunk the walker stands on
+    int2 w_pg = make_int2(0, 0);                                  // its two page ids (requested one chunk ahead)
+    int tiles_issued = 0;                                         // tile stages of the chunks walked so far (ring position)
+    bool ok = true;
+    auto wait = [&](uint32_t mbar, uint32_t parity) {
+        if (!tc::mbar_wait(mbar, parity, ok ? (1u << 18) : 1u, fail)) {
+            ok = false;
+            *fail = 1;
+        }
+    };
+    auto page_ids = [&](int bb, int cc) {
+        const int32_t *bt = p.block_table + (size_t)bb * p.max_pages_per_seq + cc * 2;
+        int2 r;
+        r.x = (cc * 2 < p.max_pages_per_seq) ? __ldg(bt) : 0;
+        r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
+        return r;
+    };
+    auto walk_begin = [&]() {
+        w_b = range[1], w_head = range[2], w_chunk = range[3], w_nc = range[4], w_len = range[5];
+        w_pg = page_ids(w_b, w_chunk);
+    };
+    // Walks chunks [n_from, n_to) of the block's list, asking the copy engine for each chunk's tiles (K tiles, then V
+    // tiles, in the order the consumers need them) and / or for its record: coordinates, the scales of its tiles (K
+    // and V scales of a page and head are adjacent: one 1 KB copy per tile) and the query rows unless the group that
+    // takes the chunk still holds them from its previous chunk (same sequence and kv head).
+    auto walk = [&](int n_from, int n_to, int n_end, bool tiles, bool records) {
+        for (int n = n_from; n < n_to; ++n) {
+            const int cb = w_b, chead = w_head, cchunk = w_chunk;
+            const int n_tok = min(kStChunk, w_len - w_chunk * kStChunk);
+            const int2 cpg = w_pg;
+            // ---- the next chunk's coordinates and page ids, requested before this chunk's copies are issued
+            if (n + 1 < n_end) {
+                st_next_chunk(p, B, w_b, w_head, w_chunk, w_len, w_nc);
+                w_pg = page_ids(min(w_b, B - 1), w_chunk);
+            }
+            int page[2] = {cpg.x, cpg.y};
+            int rows16[2];
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                page[t] = (page[t] >= 0 && page[t] < p.num_pages) ? page[t] : 0;
+                const int rows = max(0, min(kStTile, n_tok - t * kStTile));
+                rows16[t] = (rows + kStTailBox - 1) / kStTailBox * kStTailBox;
+            }
+            const int n_tiles = rows16[1] > 0 ? 2 : 1;
+            if (records) {
+                const int islot = n % kStInfoSlots;
+                const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
+                wait(bar_info_empty(islot), iph ^ 1u);
+                unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
+                const uint32_t info_addr = sbase + L::kInfo0 + islot * L::kInfoBytes;
+                int *meta = reinterpret_cast<int *>(info + L::kMeta);
+                meta[0] = cb, meta[1] = chead, meta[2] = cchunk, meta[3] = n_tok, meta[4] = tiles_issued;
+                const bool need_q = !(n >= kStGroups && cchunk >= kStGroups);
+                const uint32_t q_bytes = need_q ? (uint32_t)p.G * kHeadDim * 2u : 0u;
+                tc::mbar_arrive_expect_tx(bar_info_full(islot), (uint32_t)n_tiles * 1024u + q_bytes);
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+                    if (t < n_tiles)
+                        tc::bulk_load(info_addr + L::kScales + t * 1024, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
+                                      1024u, bar_info_full(islot));
+                if (need_q)
+                    tc::bulk_load(info_addr + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes,
+                                  bar_info_full(islot));
+            }
+            if (tiles) {
+                int gi = tiles_issued;
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (rows16[t] == 0) continue;
+                        const int stage = gi % S;
+                        wait(bar_empty(stage), ((uint32_t)(gi / S) & 1u) ^ 1u);
+                        const uint32_t full = bar_full(stage);
+                        tc::mbar_arrive_expect_tx(full, (uint32_t)rows16[t] * kHeadDim);
+                        const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
+                        const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
+                        if (rows16[t] == kStTile) {
+                            tc::tma_load_2d(dst, &map_tile, 0, row0, full);
+                        } else {
+                            for (int r = 0; r < rows16[t]; r += kStTailBox)
+                                tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
+                        }
+                        ++gi;
+                    }
+                }
+            }
+            tiles_issued += 2 * n_tiles;
+        }
+    };
+    constexpr int kBarSetup = 8, kBarProducers = 9;   // named barriers (1 .. kGroups belong to the consumer groups)
+
+    if (warp == kPW && lane == 0) {
+        tc::prefetch_tensormap(&map_tile);   // (kernel parameters: nothing an earlier kernel writes)
+        tc::prefetch_tensormap(&map_tail);
         for (int i = 0; i < S; ++i) {
             tc::mbar_init(bar_full(i), 1);
             tc::mbar_init(bar_empty(i), 1);
@@ -352,199 +441,114 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         pdl_wait();
         // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order.  The work is cut
         //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.
-        const int len_first = (lane < B) ? st_chunk_len(p, lane) : 0;   // the first 32 sequences stay in registers
-        auto seq_len = [&](int base) {   // tokens of sequence base + lane that the chunks cover
-            const int b = base + lane;
-            return (base == 0) ? len_first : ((b < B) ? st_chunk_len(p, b) : 0);
+        // (a warp scan over the sequences' tile and chunk counts, 32 sequences at a time; the first 32 sequences' counts
+        // and scans stay in registers and serve both cut points)
+        struct Scan {
+            int len, nt, nc, it, ic;   // tokens covered by chunks, tiles, chunks; inclusive prefix sums of tiles and chunks over the lanes
         };
-        long long tiles_all = 0;
-        for (int base = 0; base < B; base += 32)
-            tiles_all += __reduce_add_sync(0xffffffffu, (seq_len(base) + kStTile - 1) / kStTile);
-        const long long total_tiles = tiles_all * p.Hkv;
-        // number of chunks that start before tile index x (x <= total_tiles), over all (sequence, kv head) runs in order
-        auto chunks_before = [&](long long x) {
-            long long tiles_pre = 0, chunks_pre = 0;
-            for (int base = 0; base < B; base += 32) {
-                const int len = seq_len(base);
-                const int nt = (len + kStTile - 1) / kStTile, nc = (len + kStChunk - 1) / kStChunk;
-                int it = nt, ic = nc;
+        auto scan_block = [&](int base) {
+            Scan r;
+            const int b = base + lane;
+            r.len = (b < B) ? st_chunk_len(p, b) : 0;
+            r.nt = (r.len + kStTile - 1) / kStTile;
+            r.nc = (r.len + kStChunk - 1) / kStChunk;
+            r.it = r.nt;
+            r.ic = r.nc;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int vt = __shfl_up_sync(0xffffffffu, it, o), vc = __shfl_up_sync(0xffffffffu, ic, o);
-                    if (lane >= o) it += vt, ic += vc;
-                }
-                const unsigned hit = __ballot_sync(0xffffffffu, (tiles_pre + it) * p.Hkv > x);
+            for (int o = 1; o < 32; o <<= 1) {
+                const int vt = __shfl_up_sync(0xffffffffu, r.it, o), vc = __shfl_up_sync(0xffffffffu, r.ic, o);
+                if (lane >= o) r.it += vt, r.ic += vc;
+            }
+            return r;
+        };
+        const Scan first = scan_block(0);
+        long long tiles_all = __shfl_sync(0xffffffffu, first.it, 31);
+        for (int base = 32; base < B; base += 32) tiles_all += __shfl_sync(0xffffffffu, scan_block(base).it, 31);
+        const long long total_tiles = tiles_all * p.Hkv;
+        // The cut at tile index x (x <= total_tiles): the number of chunks that start before it, over all (sequence,
+        // kv head) runs in order, and where it falls: sequence, kv head, chunk (which may be the run's chunk count:
+        // the cut then lies at the start of the next run), that sequence's chunk count and chunk tokens.
+        struct Cut {
+            long long index;
+            int b, head, chunk, nc, len;
+        };
+        auto cut_at = [&](long long x) {
+            long long tiles_pre = 0, chunks_pre = 0;
+            Cut c;
+            c.b = c.head = c.chunk = 0;
+            c.nc = 1;
+            c.len = 0;
+            for (int base = 0; base < B; base += 32) {
+                const Scan sc = (base == 0) ? first : scan_block(base);
+                const unsigned hit = __ballot_sync(0xffffffffu, (tiles_pre + sc.it) * p.Hkv > x);
                 if (hit != 0u) {
                     const int l = __ffs(hit) - 1;
-                    const int nt_l = __shfl_sync(0xffffffffu, nt, l), nc_l = __shfl_sync(0xffffffffu, nc, l);
-                    const long long tb = tiles_pre + __shfl_sync(0xffffffffu, it, l) - nt_l;
-                    const long long cb = chunks_pre + __shfl_sync(0xffffffffu, ic, l) - nc_l;
+                    const int nt_l = __shfl_sync(0xffffffffu, sc.nt, l), nc_l = __shfl_sync(0xffffffffu, sc.nc, l);
+                    const long long tb = tiles_pre + __shfl_sync(0xffffffffu, sc.it, l) - nt_l;
+                    const long long cb = chunks_pre + __shfl_sync(0xffffffffu, sc.ic, l) - nc_l;
                     const int r = (int)(x - tb * p.Hkv);             // < Hkv * nt_l
                     const int head = r / nt_l, d = r - head * nt_l;
-                    return cb * p.Hkv + (long long)head * nc_l + min(nc_l, (d + 1) / 2);
+                    c.b = base + l;
+                    c.head = head;
+                    c.chunk = min(nc_l, (d + 1) / 2);
+                    c.nc = nc_l;
+                    c.len = __shfl_sync(0xffffffffu, sc.len, l);
+                    c.index = cb * p.Hkv + (long long)head * nc_l + c.chunk;
+                    return c;
                 }
-                tiles_pre += __shfl_sync(0xffffffffu, it, 31);
-                chunks_pre += __shfl_sync(0xffffffffu, ic, 31);
+                tiles_pre += __shfl_sync(0xffffffffu, sc.it, 31);
+                chunks_pre += __shfl_sync(0xffffffffu, sc.ic, 31);
             }
-            return chunks_pre * p.Hkv;
+            c.index = chunks_pre * p.Hkv;
+            return c;
         };
-        const long long i0 = chunks_before(st_div(total_tiles * blockIdx.x, (int)gridDim.x));
-        const long long i1 = chunks_before(st_div(total_tiles * (blockIdx.x + 1), (int)gridDim.x));
-        int b0 = 0, head0 = 0, chunk0 = 0, nc0 = 1;
-        if (i1 > i0) {
-            long long prefix = 0;   // chunks of the sequences before `base`
-            for (int base = 0; base < B; base += 32) {
-                const int nc = (seq_len(base) + kStChunk - 1) / kStChunk;
-                int incl = nc;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += v;
-                }
-                const unsigned hit = __ballot_sync(0xffffffffu, (prefix + incl) * p.Hkv > i0);
-                if (hit != 0u) {
-                    const int l = __ffs(hit) - 1;
-                    const int nc_l = __shfl_sync(0xffffffffu, nc, l);
-                    const long long before = prefix + __shfl_sync(0xffffffffu, incl, l) - nc_l;
-                    const int r = (int)(i0 - before * p.Hkv);   // < Hkv * nc_l
-                    b0 = base + l;
-                    head0 = r / nc_l;
-                    chunk0 = r - head0 * nc_l;
-                    nc0 = nc_l;
-                    break;
-                }
-                prefix += __shfl_sync(0xffffffffu, incl, 31);
-            }
-        }
+        const Cut c0 = cut_at(st_div(total_tiles * blockIdx.x, (int)gridDim.x));
+        const Cut c1 = cut_at(st_div(total_tiles * (blockIdx.x + 1), (int)gridDim.x));
         if (lane == 0) {
-            range[0] = (int)(i1 - i0);
+            int b0 = c0.b, head0 = c0.head, chunk0 = c0.chunk - 1, nc0 = c0.nc, len0 = c0.len;
+            // one step from the chunk before the cut: a cut at the end of a run moves to the next run with chunks
+            if (c1.index > c0.index) st_next_chunk(p, B, b0, head0, chunk0, len0, nc0);
+            range[0] = (int)(c1.index - c0.index);
             range[1] = b0;
             range[2] = head0;
             range[3] = chunk0;
             range[4] = nc0;
+            range[5] = len0;
         }
+        __syncwarp();
     } else if (warp < kPW) {
         // rows of the query operand that belong to no head stay zero for the whole launch
         const int g = warp >> 2, gtid = tid & 127;
         unsigned char *qop = smem + L::kGroup0 + g * L::kGroupBytes + L::kQop;
         for (int i = gtid * 16; i < NS * 128; i += kStGroupThreads * 16) *reinterpret_cast<uint4 *>(qop + i) = make_uint4(0, 0, 0, 0);
-    } else if (use_table) {
-        // the second producer warp and the MMA-issue warps copy the block table while the lengths are on their way
-        pdl_wait();
-        constexpr int kCopyThreads = L::kThreads - (kPW + 1) * 32;
-        for (int i = tid - (kPW + 1) * 32; i < table_ints; i += kCopyThreads) table[i] = __ldg(p.block_table + i);
     }
+    // ---- the block's set-up barrier.  The two producer warps do not wait on it: the first one passes the range to the
+    //      second through a barrier of their own, both signal their arrival on the block's barrier and start asking for
+    //      the first chunks at once, so that those copies are in flight while the other warps are still on their way.
     tc::fence_proxy_async();
     tc::fence_before_sync();
-    __syncthreads();
+    __threadfence_block();
+    if (warp == kPW) {
+        tc::named_barrier_arrive(kBarProducers, 64);
+        tc::named_barrier_arrive(kBarSetup, L::kThreads);
+    } else if (warp == kPW + 1) {
+        tc::named_barrier(kBarProducers, 64);
+        tc::named_barrier_arrive(kBarSetup, L::kThreads);
+    } else {
+        tc::named_barrier(kBarSetup, L::kThreads);
+    }
     tc::fence_after_sync();
-    const uint32_t tmem = *tmem_slot;
+    const uint32_t tmem = (warp == kPW || warp == kPW + 1) ? 0u : *tmem_slot;   // (the producers do not touch tensor memory)
     const int cnt = range[0];
-    bool ok = true;
-    auto wait = [&](uint32_t mbar, uint32_t parity) {
-        if (!tc::mbar_wait(mbar, parity, ok ? (1u << 18) : 1u, fail)) {
-            ok = false;
-            *fail = 1;
-        }
-    };
-    int tiles_issued = 0;   // producer thread: tile stages armed so far (ring position)
 
     if (warp == kPW || warp == kPW + 1) {
         // =========================================================== producers (one thread each)
-        // warp kPW walks the block's chunks and asks for their K and V tiles; warp kPW + 1 walks the same
-        // list and asks for the chunk records (coordinates, scales, query rows).  Two threads because
-        // the rate at which one thread can hand requests to the copy engine would otherwise limit the stream.
-        const bool tile_role = warp == kPW;
+        // warp kPW walks the block's chunks and asks for their K and V tiles; warp kPW + 1 walks the same list and
+        // asks for the chunk records.  Two threads because the rate at which one thread can hand requests to the
+        // copy engine (about one per 100 ns) would otherwise limit the stream.
         if (lane == 0 && cnt > 0) {
-            pdl_wait();   // (returns at once: the earlier kernel was already waited for before the lengths were read)
-            int b = range[1], head = range[2], chunk = range[3];
-            int len = st_chunk_len(p, b);
-            int nc = (len + kStChunk - 1) / kStChunk;
-            auto page_ids = [&](int bb, int cc) {
-                int2 r;
-                if (use_table) {
-                    const int at = bb * p.max_pages_per_seq + cc * 2;
-                    r.x = (cc * 2 < p.max_pages_per_seq) ? table[at] : 0;
-                    r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? table[at + 1] : 0;
-                } else {
-                    const int32_t *bt = p.block_table + (size_t)bb * p.max_pages_per_seq + cc * 2;
-                    r.x = (cc * 2 < p.max_pages_per_seq) ? __ldg(bt) : 0;
-                    r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
-                }
-                return r;
-            };
-            const uint64_t stream_policy = tc::policy_evict_first();   // cache rows are read once per launch
-            int2 pg = page_ids(b, chunk);
-            int stage = 0;
-            uint32_t stage_ph = 0;   // parity of the stage's current use
-            for (int n = 0; n < cnt; ++n) {
-                const int cb = b, chead = head, cchunk = chunk;
-                const int n_tok = min(kStChunk, len - chunk * kStChunk);
-                const int2 cpg = pg;
-                // ---- the next chunk's coordinates and page ids, requested before this chunk's copies are issued
-                if (n + 1 < cnt) {
-                    st_next_chunk(p, B, b, head, chunk, len, nc);
-                    pg = page_ids(min(b, B - 1), chunk);
-                }
-                int page[2] = {cpg.x, cpg.y};
-                int rows16[2];
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    page[t] = (page[t] >= 0 && page[t] < p.num_pages) ? page[t] : 0;
-                    const int rows = max(0, min(kStTile, n_tok - t * kStTile));
-                    rows16[t] = (rows + kStTailBox - 1) / kStTailBox * kStTailBox;
-                }
-                const int n_tiles = rows16[1] > 0 ? 2 : 1;
-                if (!tile_role) {
-                    // ---- the chunk record: coordinates, the scales of its tiles (K and V scales of a page and head
-                    //      are adjacent: one 1 KB copy per tile), and the query rows unless the group that takes
-                    //      this chunk still holds them from its previous chunk (same sequence and kv head)
-                    const int islot = n % kStInfoSlots;
-                    const uint32_t iph = (uint32_t)(n / kStInfoSlots) & 1u;
-                    wait(bar_info_empty(islot), iph ^ 1u);
-                    unsigned char *info = smem + L::kInfo0 + islot * L::kInfoBytes;
-                    const uint32_t info_addr = sbase + L::kInfo0 + islot * L::kInfoBytes;
-                    int *meta = reinterpret_cast<int *>(info + L::kMeta);
-                    meta[0] = cb, meta[1] = chead, meta[2] = cchunk, meta[3] = n_tok, meta[4] = tiles_issued;
-                    const bool need_q = !(n >= kStGroups && cchunk >= kStGroups);
-                    const uint32_t q_bytes = need_q ? (uint32_t)p.G * kHeadDim * 2u : 0u;
-                    tc::mbar_arrive_expect_tx(bar_info_full(islot), (uint32_t)n_tiles * 1024u + q_bytes);
-#pragma unroll
-                    for (int t = 0; t < 2; ++t)
-                        if (t < n_tiles)
-                            tc::bulk_load_hint(info_addr + L::kScales + t * 1024, p.scales + scale_block_offset(page[t], chead, 0, p.Hkv),
-                                               1024u, bar_info_full(islot), stream_policy);
-                    if (need_q)
-                        tc::bulk_load(info_addr + L::kQraw, p.q + ((size_t)cb * p.Hq + (size_t)chead * p.G) * kHeadDim, q_bytes,
-                                      bar_info_full(islot));
-                    tiles_issued += 2 * n_tiles;
-                } else {
-                    // ---- the chunk's tiles, in the order the consumers need them: K tiles, then V tiles
-#pragma unroll
-                    for (int kv = 0; kv < 2; ++kv) {
-#pragma unroll
-                        for (int t = 0; t < 2; ++t) {
-                            if (rows16[t] == 0) continue;
-                            wait(bar_empty(stage), stage_ph ^ 1u);
-                            const uint32_t full = bar_full(stage);
-                            tc::mbar_arrive_expect_tx(full, (uint32_t)rows16[t] * kHeadDim);
-                            const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
-                            const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
-                            if (rows16[t] == kStTile) {
-                                tc::tma_load_2d_hint(dst, &map_tile, 0, row0, full, stream_policy);
-                            } else {
-                                for (int r = 0; r < rows16[t]; r += kStTailBox)
-                                    tc::tma_load_2d_hint(dst + r * kHeadDim, &map_tail, 0, row0 + r, full, stream_policy);
-                            }
-                            ++tiles_issued;
-                            if (++stage == S) {
-                                stage = 0;
-                                stage_ph ^= 1u;
-                            }
-                        }
-                    }
-                }
-            }
+            walk_begin();
+            walk(0, cnt, cnt, warp == kPW, warp == kPW + 1);
         }
     } else if (warp > kPW + 1) {
         // =========================================================== MMA issue for group g (one thread)
@@ -638,7 +642,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             pdl_wait();
             if (cnt > 0) {
                 int b = range[1], head = range[2];
-                int L = st_clamped_len(p, b);
+                int L = range[5] + 1;   // the chunks cover all of the sequence's tokens but the last
                 int nc = range[4];
                 int last = nc - 1 - range[3];   // list index of the pair's last chunk
                 for (int r = 0; last < cnt; ++r) {
@@ -902,7 +906,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         }
         __syncwarp();
         tc::fence_after_sync();
-        tc::tmem_dealloc(tmem, L::kTmemCols);
+        tc::tmem_dealloc(*tmem_slot, L::kTmemCols);   // (this warp allocated it; the block's last barrier lies behind)
     }
 }
 

@@ -177,22 +177,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void *tmap,
         "l"(tmap), "r"(x), "r"(y), "r"(mbar_smem)
         : "memory");
 }
-// The same copy with a cache policy for the L2 (see policy_evict_first).
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst_smem, const void *tmap, int x, int y, uint32_t mbar_smem, uint64_t policy)
+// Asks the copy engine to fetch a tensor map (a kernel parameter) ahead of its first use.
+__device__ __forceinline__ void prefetch_tensormap(const void *tmap)
 {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;\n" ::"r"(
-            dst_smem),
-        "l"(tmap), "r"(x), "r"(y), "r"(mbar_smem), "l"(policy)
-        : "memory");
-}
-// L2 policy for data that is read once: its lines are the first to be replaced, so that a long stream does not
-// push the small tables and partial results that are read again out of the L2.
-__device__ __forceinline__ uint64_t policy_evict_first()
-{
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
-    return policy;
+    asm volatile("prefetch.tensormap [%0];\n" ::"l"(tmap) : "memory");
 }
 // Untiled bulk copy global -> shared: both addresses 16-byte aligned, size a multiple of 16.
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t mbar_smem)
@@ -202,17 +190,16 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, ui
         "l"(src), "r"(bytes), "r"(mbar_smem)
         : "memory");
 }
-__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t mbar_smem, uint64_t policy)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(dst_smem),
-        "l"(src), "r"(bytes), "r"(mbar_smem), "l"(policy)
-        : "memory");
-}
 // Barrier among `count` threads (a multiple of 32) of the block, id 1..15.
 __device__ __forceinline__ void named_barrier(int id, int count)
 {
     asm volatile("bar.sync %0, %1;\n" ::"r"(id), "r"(count) : "memory");
+}
+// Signals this thread's arrival on the barrier without waiting for the others (who use named_barrier with the same
+// id and count).  A thread that arrives this way must make its earlier writes visible itself (__threadfence_block).
+__device__ __forceinline__ void named_barrier_arrive(int id, int count)
+{
+    asm volatile("bar.arrive %0, %1;\n" ::"r"(id), "r"(count) : "memory");
 }
 
 }  // namespace tc
