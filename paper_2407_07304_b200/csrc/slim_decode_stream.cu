@@ -89,8 +89,8 @@ struct StSmem {
     static constexpr uint32_t kBar = kGroup0 + kGroups * kGroupBytes;
     static constexpr int kNumBars = 2 * kStages + 2 * kInfoSlots + 4 * kGroups;
     static constexpr uint32_t kTmemSlot = kBar + kNumBars * 8;
-    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[6]: chunks of this block, first sequence / head / chunk, that sequence's chunks and chunk tokens
-    static constexpr uint32_t kFail = kRange + 32;
+    static constexpr uint32_t kRange = (kTmemSlot + 8 + 15) / 16 * 16;   // int[6]: -, the block's first sequence / head / chunk, that sequence's chunks and chunk tokens; at +32: long long[2], the global chunk indices where the range starts and ends
+    static constexpr uint32_t kFail = kRange + 48;
     static constexpr uint32_t kBytes = kFail + 16;
     static_assert(kRange % 16 == 0, "range record is read as int4-aligned ints");
     static_assert(kBytes <= 232448, "shared memory budget of one block");
@@ -204,38 +204,48 @@ __device__ __forceinline__ void st_last_token(const DecodeParams &p, int b, int 
         c[4 + i] = (float)(int)(int8_t)((pk.y >> (8 * i)) & 0xFFu);
     }
     const float lsv = __log2f(sv), rsv = st_rcp(sv), ks = sk * p.scale_log2e;
-    for (int h = 0; h < p.G; ++h) {
-        const size_t row = (size_t)b * p.Hq + (size_t)head * p.G + h;
-        if (to_out) {
-            if (kv == 1) {
-                uint32_t w[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    __nv_bfloat162 x = __floats2bfloat162_rn(c[2 * i] * sv, c[2 * i + 1] * sv);
-                    w[i] = *reinterpret_cast<uint32_t *>(&x);
-                }
-                reinterpret_cast<uint4 *>(p.out + row * kHeadDim)[l] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            continue;
-        }
-        const uint4 qv = __ldg(reinterpret_cast<const uint4 *>(p.q + row * kHeadDim) + l);
-        const uint32_t qw[4] = {qv.x, qv.y, qv.z, qv.w};
-        float dot = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            dot = fmaf(bf16_bits_to_float(qw[i] & 0xFFFFu), c[2 * i], dot);
-            dot = fmaf(bf16_bits_to_float(qw[i] >> 16), c[2 * i + 1], dot);
-        }
-#pragma unroll
-        for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // lanes 0-15: q . k codes
-        const float s = __shfl_sync(0xffffffffu, dot, 0);
-        const size_t ps = row * p.n_slots + slot;
+    if (to_out) {
+        // a sequence of one token: its softmax weight is 1 and the result is the dequantised V row
         if (kv == 1) {
-            float4 *dst = reinterpret_cast<float4 *>(p.part_o + ps * kHeadDim + 8 * l);
-            dst[0] = make_float4(c[0], c[1], c[2], c[3]);
-            dst[1] = make_float4(c[4], c[5], c[6], c[7]);
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                __nv_bfloat162 x = __floats2bfloat162_rn(c[2 * i] * sv, c[2 * i + 1] * sv);
+                w[i] = *reinterpret_cast<uint32_t *>(&x);
+            }
+            for (int h = 0; h < p.G; ++h)
+                reinterpret_cast<uint4 *>(p.out + ((size_t)b * p.Hq + (size_t)head * p.G + h) * kHeadDim)[l] = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (lane == 0) *reinterpret_cast<float2 *>(p.part_ml + ps * 2) = make_float2(fmaf(s, ks, lsv), rsv);
+        return;
+    }
+    const size_t row0 = (size_t)b * p.Hq + (size_t)head * p.G;
+    for (int h0 = 0; h0 < p.G; h0 += 8) {
+        // eight heads' query rows are requested together (one round trip instead of eight)
+        uint4 qv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            qv[i] = (h0 + i < p.G) ? __ldg(reinterpret_cast<const uint4 *>(p.q + (row0 + h0 + i) * kHeadDim) + l) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (h0 + i >= p.G) break;
+            const uint32_t qw[4] = {qv[i].x, qv[i].y, qv[i].z, qv[i].w};
+            float dot = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                dot = fmaf(bf16_bits_to_float(qw[k] & 0xFFFFu), c[2 * k], dot);
+                dot = fmaf(bf16_bits_to_float(qw[k] >> 16), c[2 * k + 1], dot);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // lanes 0-15: q . k codes
+            const float s = __shfl_sync(0xffffffffu, dot, 0);
+            const size_t ps = (row0 + h0 + i) * p.n_slots + slot;
+            if (kv == 1) {
+                float4 *dst = reinterpret_cast<float4 *>(p.part_o + ps * kHeadDim + 8 * l);
+                dst[0] = make_float4(c[0], c[1], c[2], c[3]);
+                dst[1] = make_float4(c[4], c[5], c[6], c[7]);
+            }
+            if (lane == 0) *reinterpret_cast<float2 *>(p.part_ml + ps * 2) = make_float2(fmaf(s, ks, lsv), rsv);
+        }
     }
 }
 
@@ -338,6 +348,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         r.y = (cc * 2 + 1 < p.max_pages_per_seq) ? __ldg(bt + 1) : 0;
         return r;
     };
+    const uint64_t stream_policy = tc::policy_evict_first();   // cache rows are read once per launch
     auto walk_begin = [&]() {
         w_b = range[1], w_head = range[2], w_chunk = range[3], w_nc = range[4], w_len = range[5];
         w_pg = page_ids(w_b, w_chunk);
@@ -399,10 +410,10 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                         const int row0 = ((page[t] * p.Hkv + chead) * 2 + kv) * kPageTokens;
                         const uint32_t dst = sbase + (uint32_t)stage * kStTileBytes;
                         if (rows16[t] == kStTile) {
-                            tc::tma_load_2d(dst, &map_tile, 0, row0, full);
+                            tc::tma_load_2d_hint(dst, &map_tile, 0, row0, full, stream_policy);
                         } else {
                             for (int r = 0; r < rows16[t]; r += kStTailBox)
-                                tc::tma_load_2d(dst + r * kHeadDim, &map_tail, 0, row0 + r, full);
+                                tc::tma_load_2d_hint(dst + r * kHeadDim, &map_tail, 0, row0 + r, full, stream_policy);
                         }
                         ++gi;
                     }
@@ -434,51 +445,73 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
         tc::mbar_init_fence();
         *fail = 0;
     }
-    if (warp == kPW) {
-        tc::tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
+    if (warp == kPW) tc::tmem_alloc(smem_u32(tmem_slot), L::kTmemCols);
+    if (warp == kPW || warp == kPW + 1) {
         // Up to here the block may run beside the kernel before it in the stream (the same step's
         // slim_kv_append); from here on it reads what earlier kernels may have written.
         pdl_wait();
         // ---- this block's contiguous range of chunks, in (sequence, kv head, chunk) order.  The work is cut
-        //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.
-        // (a warp scan over the sequences' tile and chunk counts, 32 sequences at a time; the first 32 sequences' counts
-        // and scans stay in registers and serve both cut points)
-        struct Scan {
-            int len, nt, nc, it, ic;   // tokens covered by chunks, tiles, chunks; inclusive prefix sums of tiles and chunks over the lanes
-        };
-        auto scan_block = [&](int base) {
-            Scan r;
-            const int b = base + lane;
-            r.len = (b < B) ? st_chunk_len(p, b) : 0;
-            r.nt = (r.len + kStTile - 1) / kStTile;
-            r.nc = (r.len + kStChunk - 1) / kStChunk;
-            r.it = r.nt;
-            r.ic = r.nc;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int vt = __shfl_up_sync(0xffffffffu, r.it, o), vc = __shfl_up_sync(0xffffffffu, r.ic, o);
-                if (lane >= o) r.it += vt, r.ic += vc;
-            }
-            return r;
-        };
-        const Scan first = scan_block(0);
-        long long tiles_all = __shfl_sync(0xffffffffu, first.it, 31);
-        for (int base = 32; base < B; base += 32) tiles_all += __shfl_sync(0xffffffffu, scan_block(base).it, 31);
-        const long long total_tiles = tiles_all * p.Hkv;
-        // The cut at tile index x (x <= total_tiles): the number of chunks that start before it, over all (sequence,
+        //      by 128-token tiles (what a chunk costs) and the cut points are moved up to chunk starts.  The first
+        //      producer warp finds where the range starts, the second where it ends, at the same time.
+        // The cut at tile index x (x <= total tiles): the number of chunks that start before it, over all (sequence,
         // kv head) runs in order, and where it falls: sequence, kv head, chunk (which may be the run's chunk count:
         // the cut then lies at the start of the next run), that sequence's chunk count and chunk tokens.
         struct Cut {
             long long index;
             int b, head, chunk, nc, len;
         };
-        auto cut_at = [&](long long x) {
+        Cut cut;
+        cut.b = cut.head = cut.chunk = cut.len = 0;
+        cut.nc = 1;
+        const int which = warp - kPW;   // 0: the range's start, 1: its end
+        const int len_first = (lane < B) ? st_chunk_len(p, lane) : 0;   // tokens of the first 32 sequences that chunks cover
+        const int len_u = __shfl_sync(0xffffffffu, len_first, 0);
+        bool uniform = __all_sync(0xffffffffu, lane >= B || len_first == len_u);
+        for (int base = 32; base < B && uniform; base += 32)
+            uniform = __all_sync(0xffffffffu, base + lane >= B || st_chunk_len(p, base + lane) == len_u);
+        if (uniform) {
+            // every sequence has the same length (a batch decoded in lockstep): the cut has a closed form
+            const int nt = (len_u + kStTile - 1) / kStTile, nc = (len_u + kStChunk - 1) / kStChunk;
+            const long long pairs = (long long)B * p.Hkv;
+            const long long x = st_div(pairs * nt * (blockIdx.x + which), (int)gridDim.x);
+            cut.index = pairs * nc;
+            if (x < pairs * nt) {
+                const long long pair = st_div(x, nt);
+                const int d = (int)(x - pair * nt);
+                cut.b = (int)st_div(pair, p.Hkv);
+                cut.head = (int)(pair - (long long)cut.b * p.Hkv);
+                cut.chunk = min(nc, (d + 1) / 2);
+                cut.nc = nc;
+                cut.len = len_u;
+                cut.index = pair * nc + cut.chunk;
+            }
+        } else {
+            // a warp scan over the sequences' tile and chunk counts, 32 sequences at a time
+            struct Scan {
+                int len, nt, nc, it, ic;   // tokens covered by chunks, tiles, chunks; inclusive prefix sums of tiles and chunks over the lanes
+            };
+            auto scan_block = [&](int base) {
+                Scan r;
+                const int b = base + lane;
+                r.len = (base == 0) ? len_first : ((b < B) ? st_chunk_len(p, b) : 0);
+                r.nt = (r.len + kStTile - 1) / kStTile;
+                r.nc = (r.len + kStChunk - 1) / kStChunk;
+                r.it = r.nt;
+                r.ic = r.nc;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int vt = __shfl_up_sync(0xffffffffu, r.it, o), vc = __shfl_up_sync(0xffffffffu, r.ic, o);
+                    if (lane >= o) r.it += vt, r.ic += vc;
+                }
+                return r;
+            };
+            const Scan first = scan_block(0);
+            long long tiles_all = __shfl_sync(0xffffffffu, first.it, 31);
+            for (int base = 32; base < B; base += 32) tiles_all += __shfl_sync(0xffffffffu, scan_block(base).it, 31);
+            const long long x = st_div(tiles_all * p.Hkv * (blockIdx.x + which), (int)gridDim.x);
             long long tiles_pre = 0, chunks_pre = 0;
-            Cut c;
-            c.b = c.head = c.chunk = 0;
-            c.nc = 1;
-            c.len = 0;
-            for (int base = 0; base < B; base += 32) {
+            bool found = false;
+            for (int base = 0; base < B && !found; base += 32) {
                 const Scan sc = (base == 0) ? first : scan_block(base);
                 const unsigned hit = __ballot_sync(0xffffffffu, (tiles_pre + sc.it) * p.Hkv > x);
                 if (hit != 0u) {
@@ -488,58 +521,58 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                     const long long cb = chunks_pre + __shfl_sync(0xffffffffu, sc.ic, l) - nc_l;
                     const int r = (int)(x - tb * p.Hkv);             // < Hkv * nt_l
                     const int head = r / nt_l, d = r - head * nt_l;
-                    c.b = base + l;
-                    c.head = head;
-                    c.chunk = min(nc_l, (d + 1) / 2);
-                    c.nc = nc_l;
-                    c.len = __shfl_sync(0xffffffffu, sc.len, l);
-                    c.index = cb * p.Hkv + (long long)head * nc_l + c.chunk;
-                    return c;
+                    cut.b = base + l;
+                    cut.head = head;
+                    cut.chunk = min(nc_l, (d + 1) / 2);
+                    cut.nc = nc_l;
+                    cut.len = __shfl_sync(0xffffffffu, sc.len, l);
+                    cut.index = cb * p.Hkv + (long long)head * nc_l + cut.chunk;
+                    found = true;
+                } else {
+                    tiles_pre += __shfl_sync(0xffffffffu, sc.it, 31);
+                    chunks_pre += __shfl_sync(0xffffffffu, sc.ic, 31);
                 }
-                tiles_pre += __shfl_sync(0xffffffffu, sc.it, 31);
-                chunks_pre += __shfl_sync(0xffffffffu, sc.ic, 31);
             }
-            c.index = chunks_pre * p.Hkv;
-            return c;
-        };
-        const Cut c0 = cut_at(st_div(total_tiles * blockIdx.x, (int)gridDim.x));
-        const Cut c1 = cut_at(st_div(total_tiles * (blockIdx.x + 1), (int)gridDim.x));
-        if (lane == 0) {
-            int b0 = c0.b, head0 = c0.head, chunk0 = c0.chunk - 1, nc0 = c0.nc, len0 = c0.len;
-            // one step from the chunk before the cut: a cut at the end of a run moves to the next run with chunks
-            if (c1.index > c0.index) st_next_chunk(p, B, b0, head0, chunk0, len0, nc0);
-            range[0] = (int)(c1.index - c0.index);
-            range[1] = b0;
-            range[2] = head0;
-            range[3] = chunk0;
-            range[4] = nc0;
-            range[5] = len0;
+            if (!found) cut.index = chunks_pre * p.Hkv;
         }
-        __syncwarp();
+        long long *cut_index = reinterpret_cast<long long *>(smem + L::kRange + 32);
+        if (lane == 0) {
+            cut_index[which] = cut.index;
+            if (which == 0) {
+                // one step from the chunk before the cut: a cut at the end of a run moves to the next run with chunks
+                int b0 = cut.b, head0 = cut.head, chunk0 = cut.chunk - 1, nc0 = cut.nc, len0 = cut.len;
+                st_next_chunk(p, B, b0, head0, chunk0, len0, nc0);
+                range[1] = min(b0, B - 1);   // (beyond the last sequence only when the range is empty)
+                range[2] = head0;
+                range[3] = chunk0;
+                range[4] = nc0;
+                range[5] = len0;
+            }
+        }
+        // the two warps exchange what they found
+        __threadfence_block();
+        tc::named_barrier(kBarProducers, 64);
     } else if (warp < kPW) {
         // rows of the query operand that belong to no head stay zero for the whole launch
         const int g = warp >> 2, gtid = tid & 127;
         unsigned char *qop = smem + L::kGroup0 + g * L::kGroupBytes + L::kQop;
         for (int i = gtid * 16; i < NS * 128; i += kStGroupThreads * 16) *reinterpret_cast<uint4 *>(qop + i) = make_uint4(0, 0, 0, 0);
     }
-    // ---- the block's set-up barrier.  The two producer warps do not wait on it: the first one passes the range to the
-    //      second through a barrier of their own, both signal their arrival on the block's barrier and start asking for
-    //      the first chunks at once, so that those copies are in flight while the other warps are still on their way.
+    // ---- the block's set-up barrier.  The two producer warps do not wait on it (they have exchanged the range through
+    //      a barrier of their own): they signal their arrival and start asking for the first chunks at once, so that
+    //      those copies are in flight while the other warps are still on their way.
     tc::fence_proxy_async();
     tc::fence_before_sync();
     __threadfence_block();
-    if (warp == kPW) {
-        tc::named_barrier_arrive(kBarProducers, 64);
-        tc::named_barrier_arrive(kBarSetup, L::kThreads);
-    } else if (warp == kPW + 1) {
-        tc::named_barrier(kBarProducers, 64);
+    if (warp == kPW || warp == kPW + 1) {
         tc::named_barrier_arrive(kBarSetup, L::kThreads);
     } else {
         tc::named_barrier(kBarSetup, L::kThreads);
     }
     tc::fence_after_sync();
     const uint32_t tmem = (warp == kPW || warp == kPW + 1) ? 0u : *tmem_slot;   // (the producers do not touch tensor memory)
-    const int cnt = range[0];
+    const long long *cut_index_all = reinterpret_cast<const long long *>(smem + L::kRange + 32);
+    const int cnt = (int)(cut_index_all[1] - cut_index_all[0]);
 
     if (warp == kPW || warp == kPW + 1) {
         // =========================================================== producers (one thread each)

@@ -182,6 +182,24 @@ __device__ __forceinline__ void prefetch_tensormap(const void *tmap)
 {
     asm volatile("prefetch.tensormap [%0];\n" ::"l"(tmap) : "memory");
 }
+// The same copy with a cache policy for the L2 (see policy_evict_first).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst_smem, const void *tmap, int x, int y, uint32_t mbar_smem, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;\n" ::"r"(
+            dst_smem),
+        "l"(tmap), "r"(x), "r"(y), "r"(mbar_smem), "l"(policy)
+        : "memory");
+}
+// L2 policy for data that is read once: its lines are the first to be replaced, so that a long stream does not
+// push what is read again (the kernel's own instructions, the lengths and page table, the partial results) out of
+// the L2.
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(policy));
+    return policy;
+}
 // Untiled bulk copy global -> shared: both addresses 16-byte aligned, size a multiple of 16.
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t mbar_smem)
 {
