@@ -197,6 +197,32 @@ int slim_attn_decode_merge(const slim_cache_t *cache, void *out,
                            const void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Decode attention with the keys of a sequence spread over several devices
+ * (Section 2.3: the heads, and where there are fewer kv heads than devices the
+ * key range, are split across workers and combined afterwards; in Eq. 1 the
+ * batch, the heads and the tokens are plain factors).  Each device holds a
+ * part of every sequence's tokens in a cache of its own (kv_len[b] = the tokens
+ * it holds, possibly 0) and calls slim_attn_decode_partial, which is
+ * slim_attn_decode without the final normalisation: for each (sequence, query
+ * head) row it leaves the merged partial of the device's keys,
+ *
+ *   partial  device fp32 [B][Hq][SLIM_PARTIAL_FLOATS]: O[128] = sum_j 2^(s'_j - M) v^_j over the device's keys,
+ *            then M (log2 units; -inf for a row without keys) and l = sum_j 2^(s'_j - M); 16-byte aligned.
+ *
+ * The devices exchange these rows (for 32 rows 17 KB per device) and every one
+ * that needs the result calls slim_attn_merge_partials on the n_sets sets laid
+ * out back to back: M = max M_r, l = sum l_r 2^(M_r - M),
+ * o = sum O_r 2^(M_r - M) / l, written as bf16 [B][Hq][128].  The exchange itself
+ * is the caller's (one all-gather); no kernel of this library reads another
+ * device's memory.  Other arguments as for slim_attn_decode.
+ */
+#define SLIM_PARTIAL_FLOATS 132
+int slim_attn_decode_partial(const slim_cache_t *cache, const void *q, float *partial,
+                             const int32_t *kv_len, int32_t B, int32_t max_kv, int32_t Hq, float sm_scale,
+                             void *workspace, size_t workspace_bytes, void *stream);
+int slim_attn_merge_partials(const float *partials, int32_t n_sets, void *out, int32_t B, int32_t Hq, void *stream);
+
+/*
  * One decode step in one call: the new token of every sequence is quantised into
  * the cache (exactly as slim_kv_append does, Section 2.2) at position
  * kv_len[b] - 1 and decode attention runs over all kv_len[b] tokens, the new one

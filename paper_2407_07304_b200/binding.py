@@ -26,7 +26,7 @@ PAGE_TOKENS = 128
 EXPORTS = (
     "slim_kv_append", "slim_attn_prefill", "slim_attn_prefill_two_pass", "slim_attn_decode", "slim_attn_decode_split",
     "slim_attn_decode_merge", "slim_attn_decode_static", "slim_static_status", "slim_static_reset",
-    "slim_static_selftest_timeout", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
+    "slim_static_selftest_timeout", "slim_attn_decode_partial", "slim_attn_merge_partials", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
     "slim_version",
 )
@@ -86,6 +86,10 @@ def lib():
         for name in ("slim_static_status", "slim_static_reset", "slim_static_selftest_timeout"):
             getattr(L, name).argtypes = [P]
             getattr(L, name).restype = ctypes.c_int
+        L.slim_attn_decode_partial.argtypes = [CP, P, P, P, I, I, I, F, P, Z, P]
+        L.slim_attn_decode_partial.restype = ctypes.c_int
+        L.slim_attn_merge_partials.argtypes = [P, I, P, I, I, P]
+        L.slim_attn_merge_partials.restype = ctypes.c_int
         L.slim_decode_step.argtypes = [CP, P, P, P, P, P, I, I, I, F, P, Z, P]
         L.slim_decode_step.restype = ctypes.c_int
         L.slim_decode_step_host.argtypes = [CP, P, P, P, P, P, Z, P, I, I, I, F, P, Z, P]
@@ -210,6 +214,22 @@ def slim_attn_decode_static(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, stre
     rc = lib().slim_attn_decode_static(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(kv_len), B, max_kv, Hq,
                                        sm_scale, _stream(stream))
     _check(rc, "slim_attn_decode_static")
+
+
+PARTIAL_FLOATS = 132   # fp32 per (sequence, query head) row of slim_attn_decode_partial: O[128], M, l, padding
+
+
+def slim_attn_decode_partial(cache, q, partial, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None):
+    """slim_attn_decode over the part of the keys this device holds, without the final normalisation:
+    partial fp32 [B, Hq, PARTIAL_FLOATS] receives every row's merged (O, M, l)."""
+    rc = lib().slim_attn_decode_partial(ctypes.byref(cache.struct), _ptr(q), _ptr(partial), _ptr(kv_len), B, max_kv, Hq,
+                                        sm_scale, _ptr(workspace), _nbytes(workspace), _stream(stream))
+    _check(rc, "slim_attn_decode_partial")
+
+
+def slim_attn_merge_partials(partials, n_sets, out, B, Hq, stream=None):
+    """Final merge of n_sets sets of row partials (fp32 [n_sets, B, Hq, PARTIAL_FLOATS]) into bf16 out [B, Hq, 128]."""
+    _check(lib().slim_attn_merge_partials(_ptr(partials), n_sets, _ptr(out), B, Hq, _stream(stream)), "slim_attn_merge_partials")
 
 
 def slim_static_status(stream=None):

@@ -19,9 +19,12 @@ int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, c
 int launch_decode_split(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, const int32_t *kv_len,
                         int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
-                        const void *workspace, cudaStream_t stream);
+                        const void *workspace, cudaStream_t stream, float *raw = nullptr);
 int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, void *out,
                   const int32_t *kv_len, int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
+int launch_decode_partial(const slim_cache_t *c, const void *q, float *partial, const int32_t *kv_len, int B, int max_kv, int Hq,
+                          float sm_scale, void *workspace, cudaStream_t stream);
+int launch_merge_partials(const float *parts, int R, int rows, void *out, cudaStream_t stream);
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                       int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass);
@@ -139,6 +142,28 @@ SLIM_EXPORT int slim_attn_decode(const slim_cache_t *cache, const void *q, void 
     if (q == nullptr || out == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
     if (((uintptr_t)q & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
     return launch_decode(cache, q, nullptr, nullptr, out, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_attn_decode_partial(const slim_cache_t *cache, const void *q, float *partial, const int32_t *kv_len,
+                                         int32_t B, int32_t max_kv, int32_t Hq, float sm_scale, void *workspace,
+                                         size_t workspace_bytes, void *stream)
+{
+    bool launch;
+    int rc = check_decode(cache, B, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (q == nullptr || partial == nullptr || kv_len == nullptr) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)partial & 15)) return SLIM_ERR_INVALID_ARG;
+    return launch_decode_partial(cache, q, partial, kv_len, B, max_kv, Hq, sm_scale, workspace, (cudaStream_t)stream);
+}
+
+SLIM_EXPORT int slim_attn_merge_partials(const float *partials, int32_t n_sets, void *out, int32_t B, int32_t Hq, void *stream)
+{
+    if (n_sets < 0 || B < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (B == 0) return SLIM_OK;
+    if (partials == nullptr || out == nullptr || n_sets == 0) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)partials & 15) || ((uintptr_t)out & 15)) return SLIM_ERR_INVALID_ARG;
+    if ((long long)B * Hq > 0x7FFFFFFFLL / SLIM_PARTIAL_FLOATS) return SLIM_ERR_UNSUPPORTED;
+    return launch_merge_partials(partials, n_sets, B * Hq, out, (cudaStream_t)stream);
 }
 
 SLIM_EXPORT int slim_decode_step(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new, void *out,

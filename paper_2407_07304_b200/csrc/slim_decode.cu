@@ -33,7 +33,7 @@ __device__ __forceinline__ int merge_row_partials(int len, int cap_tokens)
 template <int kMergeGroups>
 __global__ void __launch_bounds__(kMergeGroups * kHeadDim)
 slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
-                         const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
+                         const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ raw,
                          int B, int Hq, int n_slots, int cap_tokens)
 {
     constexpr int kMergeThreads = kMergeGroups * kHeadDim;
@@ -92,9 +92,24 @@ slim_decode_merge_kernel(const float *__restrict__ part_o, const float *__restri
         float o = acc_s[0][d];
 #pragma unroll
         for (int i = 1; i < kMergeGroups; ++i) o += acc_s[i][d];
+        if (raw != nullptr) {
+            // the row's merged partial instead of its normalised result (the keys are split over several devices)
+            float *dst = raw + (size_t)row * SLIM_PARTIAL_FLOATS;
+            dst[d] = (nc > 0) ? o : 0.f;
+            if (d == 0) dst[kHeadDim] = (nc > 0) ? M : -INFINITY, dst[kHeadDim + 1] = (nc > 0) ? l : 0.f;
+            return;
+        }
         const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
         out[(size_t)row * kHeadDim + d] = __float2bfloat16_rn(o * inv);
     }
+}
+
+// A row's merged partial (what slim_attn_decode_partial returns): O relative to M, then M and l; a lane owns four dims.
+__device__ __forceinline__ void store_raw_partial(float *raw, int row, int lane, float4 o, float M, float l)
+{
+    float *dst = raw + (size_t)row * SLIM_PARTIAL_FLOATS;
+    reinterpret_cast<float4 *>(dst)[lane] = o;
+    if (lane == 0) *reinterpret_cast<float2 *>(dst + kHeadDim) = make_float2(M, l);
 }
 
 // A 16-byte load past the L1 cache that the compiler keeps where it is written (the merge kernels request a
@@ -115,7 +130,7 @@ constexpr int kMergeWarpBatch = 16;
 constexpr int kMergeWarpsPerBlock = 8;
 __global__ void __launch_bounds__(kMergeWarpsPerBlock * 32)
 slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
-                              const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
+                              const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ raw,
                               int B, int Hq, int n_slots, int cap_tokens)
 {
     const int lane = threadIdx.x & 31;
@@ -153,6 +168,10 @@ slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__r
             }
         }
     }
+    if (raw != nullptr) {
+        store_raw_partial(raw, row, lane, nc > 0 ? acc : make_float4(0.f, 0.f, 0.f, 0.f), nc > 0 ? M : -INFINITY, nc > 0 ? l : 0.f);
+        return;
+    }
     const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
     uint2 packed;
@@ -167,7 +186,7 @@ slim_decode_merge_warp_kernel(const float *__restrict__ part_o, const float *__r
 template <int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
-                               const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out,
+                               const int32_t *__restrict__ kv_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ raw,
                                int B, int Hq, int n_slots, int cap_tokens)
 {
     __shared__ float4 acc_s[kWarps][32];
@@ -222,6 +241,10 @@ slim_decode_merge_block_kernel(const float *__restrict__ part_o, const float *__
             r.y = fmaf(a.y, f, r.y);
             r.z = fmaf(a.z, f, r.z);
             r.w = fmaf(a.w, f, r.w);
+        }
+        if (raw != nullptr) {
+            store_raw_partial(raw, row, lane, nc > 0 ? r : make_float4(0.f, 0.f, 0.f, 0.f), nc > 0 ? M : -INFINITY, nc > 0 ? l : 0.f);
+            return;
         }
         const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
         __nv_bfloat162 lo = __floats2bfloat162_rn(r.x * inv, r.y * inv), hi = __floats2bfloat162_rn(r.z * inv, r.w * inv);
@@ -280,7 +303,7 @@ int launch_decode_split(const slim_cache_t *c, const void *q, const void *k_new,
 }
 
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
-                        const void *workspace, cudaStream_t stream);
+                        const void *workspace, cudaStream_t stream, float *raw = nullptr);
 
 // Decode attention.  With k_new / v_new the split kernel first quantises every sequence's new token into slot
 // kv_len - 1 of the cache (the one-call decode step).  Where a (sequence, kv head) has few partials the split
@@ -306,7 +329,7 @@ int launch_decode(const slim_cache_t *c, const void *q, const void *k_new, const
 }
 
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
-                        const void *workspace, cudaStream_t stream)
+                        const void *workspace, cudaStream_t stream, float *raw)
 {
     int C;
     const DecodeParams p = make_params(c, nullptr, kv_len, B, max_kv, Hq, 1.f, const_cast<void *>(workspace), C);
@@ -316,18 +339,71 @@ int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len,
     __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(out);
     if (p.n_slots >= 32 && p.n_slots <= 16 * kMergeWarpBatch) {
         if (p.n_slots <= 4 * kMergeWarpBatch)
-            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<4>, dim3(rows), dim3(128), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<4>, dim3(rows), dim3(128), 0, stream, po, pm, kv_len, o, raw, B, Hq, p.n_slots, cap));
         else if (p.n_slots <= 8 * kMergeWarpBatch)
-            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<8>, dim3(rows), dim3(256), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<8>, dim3(rows), dim3(256), 0, stream, po, pm, kv_len, o, raw, B, Hq, p.n_slots, cap));
         else
-            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<16>, dim3(rows), dim3(512), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
+            SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_block_kernel<16>, dim3(rows), dim3(512), 0, stream, po, pm, kv_len, o, raw, B, Hq, p.n_slots, cap));
     } else if (p.n_slots >= 32) {
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, po, pm, kv_len, o, B, Hq, p.n_slots, cap));
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_kernel<4>, dim3(rows), dim3(4 * kHeadDim), 0, stream, po, pm, kv_len, o, raw, B, Hq, p.n_slots, cap));
     } else {
         const int blocks = (rows + kMergeWarpsPerBlock - 1) / kMergeWarpsPerBlock;
-        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_warp_kernel, dim3(blocks), dim3(kMergeWarpsPerBlock * 32), 0, stream, po, pm, kv_len, o, B, Hq,
+        SLIM_CUDA_TRY(launch_pdl(slim_decode_merge_warp_kernel, dim3(blocks), dim3(kMergeWarpsPerBlock * 32), 0, stream, po, pm, kv_len, o, raw, B, Hq,
                                  p.n_slots, cap));
     }
+    return SLIM_OK;
+}
+
+// Decode attention over a part of every sequence's keys: split pass, then the merge pass leaves each row's merged
+// partial (O, M, l) instead of the normalised result.
+int launch_decode_partial(const slim_cache_t *c, const void *q, float *partial, const int32_t *kv_len, int B, int max_kv, int Hq,
+                          float sm_scale, void *workspace, cudaStream_t stream)
+{
+    int C;
+    DecodeParams p = make_params(c, q, kv_len, B, max_kv, Hq, sm_scale, workspace, C);
+    if (p.n_chunks > 0) {
+        const int rc = launch_decode_split_stream(c, p, B, stream);
+        if (rc != SLIM_OK) return rc;
+    }
+    return launch_decode_merge(c, nullptr, kv_len, B, max_kv, Hq, workspace, stream, partial);
+}
+
+// Final merge over R sets of row partials (one set per device that holds a part of the keys):
+//   M = max M_r;  l = sum l_r 2^(M_r - M);  o = sum O_r 2^(M_r - M) / l.   One warp per row, a lane owns four dims.
+__global__ void __launch_bounds__(256)
+slim_merge_partials_kernel(const float *__restrict__ parts, int R, int rows, __nv_bfloat16 *__restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    float M = -INFINITY;
+    for (int r = 0; r < R; ++r) M = fmaxf(M, __ldg(parts + ((size_t)r * rows + row) * SLIM_PARTIAL_FLOATS + kHeadDim));
+    float l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int r = 0; r < R; ++r) {
+        const float *src = parts + ((size_t)r * rows + row) * SLIM_PARTIAL_FLOATS;
+        const float2 ml = __ldg(reinterpret_cast<const float2 *>(src + kHeadDim));
+        if (ml.x == -INFINITY) continue;   // a device whose part of this sequence is empty
+        const float w = exp2f(ml.x - M);
+        const float4 o = __ldg(reinterpret_cast<const float4 *>(src) + lane);
+        l = fmaf(ml.y, w, l);
+        acc.x = fmaf(o.x, w, acc.x);
+        acc.y = fmaf(o.y, w, acc.y);
+        acc.z = fmaf(o.z, w, acc.z);
+        acc.w = fmaf(o.w, w, acc.w);
+    }
+    const float inv = (l > 0.f) ? 1.f / l : 0.f;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<uint32_t *>(&lo);
+    packed.y = *reinterpret_cast<uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(out + (size_t)row * kHeadDim + lane * 4) = packed;
+}
+
+int launch_merge_partials(const float *parts, int R, int rows, void *out, cudaStream_t stream)
+{
+    slim_merge_partials_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(parts, R, rows, static_cast<__nv_bfloat16 *>(out));
+    SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;
 }
 

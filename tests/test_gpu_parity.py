@@ -197,6 +197,42 @@ def test_c5_full_sampled():
     _check(workloads.make_workload(5), prefill_rows=24, decode_steps={0, 31, 63})
 
 
+# ---------------------------------------------------------------- decode spread over several ranks
+@pytest.mark.parametrize("index,shrink,world", [(4, 8, 8), (4, 8, 2), (2, 8, 4), (5, 32, 8), (5, 32, 4), (5, 32, 2), (4, 1, 8), (5, 1, 8)])
+def test_sharded_decode_every_rank_in_turn(index, shrink, world):
+    # The ranks of a plan run one after the other on this GPU: every kernel reads only its own rank's cache (the rank's
+    # kv heads, and in key-range mode its part of every sequence), and the exchange of the row partials, an all-gather
+    # between GPUs, is a torch.stack here.  Workload 4: kv heads over ranks; workload 5 (2 kv heads): key ranges.
+    from paper_2407_07304_b200.shard import ShardPlan, ShardedLayer
+    w = workloads.make_workload(index, shrink=shrink)
+    lens = [w.total_len(b) - w.decode_steps + 1 for b in range(w.B)]
+    plan = ShardPlan(w.Hq, w.Hkv, lens, world)
+    q = w.q_decode[0].cuda()
+    out = torch.zeros_like(q)
+    layers = [ShardedLayer(w, plan, r) for r in range(world)]
+    for layer in layers:
+        layer.fill()
+    if plan.mode == "heads":
+        for layer in layers:
+            out[:, layer.shard.q_heads.start:layer.shard.q_heads.stop] = layer.decode(q)
+    else:
+        for head in range(w.Hkv):
+            group = sorted((l for l in layers if layer_head(l) == head), key=lambda l: l.shard.part)
+            sets = torch.stack([l.partial_step(q).clone() for l in group])
+            res = group[0].finish(sets)
+            out[:, group[0].shard.q_heads.start:group[0].shard.q_heads.stop] = res
+    torch.cuda.synchronize()
+    oc = _oracle_cache(w)
+    rows = range(w.B) if shrink > 1 else range(min(w.B, 4))
+    for b in rows:
+        want = so.attention(bf16_bits(w.q_decode[0, b:b + 1]), *oc[b], lens[b], w.sm_scale)
+        _assert_close(out[b:b + 1], want, f"{w.name} over {world} ranks, seq {b}")
+
+
+def layer_head(layer):
+    return layer.shard.kv_heads.start
+
+
 # ---------------------------------------------------------------- edge cases
 def _custom(B, Hq, Hkv, prefill, bulk, steps, seed):
     g = torch.Generator().manual_seed(seed)
