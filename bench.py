@@ -194,6 +194,47 @@ class CacheCopy:
         self.cache, self.ws_decode = cache, ws_decode
 
 
+def timed_blocks(fn, steps, min_ms, stream, barrier, world, dev):
+    """Times blocks of exactly `steps` calls of fn, each block between two CUDA events on the launching stream and
+    bracketed by a barrier + synchronize, until at least min_ms of device time are covered (at least one block).
+    Returns the per-block times (each the max over ranks), in ms."""
+    import torch
+    blocks, total = [], 0.0
+    while True:
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        barrier()
+        ms = max_over_ranks(ms, world, dev)     # every rank sees the same number, so every rank stops together
+        blocks.append(ms)
+        total += ms
+        if total >= min_ms or len(blocks) >= 2000:
+            return blocks
+
+
+def stored_traffic():
+    """DRAM bytes per launch of the step's kernel from the ncu capture summarised under profiles/, or None when the
+    kernel's source has changed since that capture (the summary records the hash of the source it was taken on)."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", "decode_stream_workload2.md")
+    src = os.path.join(ROOT, "paper_2407_07304_b200", "csrc", "slim_decode_stream.cu")
+    try:
+        text = open(path).read()
+        digest = hashlib.sha1(open(src, "rb").read()).hexdigest()[:12]
+    except OSError:
+        return None
+    m = re.search(r"traffic_bytes_per_launch:\s*([0-9.eE+]+)\s+kernel_source_sha1:\s*([0-9a-f]+)", text)
+    if not m or m.group(2) != digest:
+        return None
+    return float(m.group(1))
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -211,6 +252,12 @@ def run_ours(args, rank, world, local_rank):
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.shard:
+        run_sharded(args, rank, world, dev, barrier)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     w = workloads.make_workload(2)
     B, Hq, Hkv, ctx = w.B, w.Hq, w.Hkv, w.bulk_len[0]
@@ -236,21 +283,9 @@ def run_ours(args, rank, world, local_rank):
     stream = torch.cuda.current_stream()
 
     def step(i):
-        # one call, one kernel: it quantises the new token's K/V rows into the cache before it reads them, streams
-        # the cache once and merges its own partial results as its blocks finish
+        # one call, one kernel: it quantises the new token's K/V rows into the cache, attends over them from registers,
+        # streams the rest of the cache once and merges its own partial results as its blocks finish
         slim.slim_decode_step(runs[i % N_ROT].cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
-
-    def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(steps):
-            fn(i)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        barrier()
-        return max_over_ranks(ms, world, dev)
 
     for i in range(max(3, args.warmup)):
         step(i)
@@ -258,13 +293,16 @@ def run_ours(args, rank, world, local_rank):
     if sampler:
         sampler.start()
         time.sleep(0.1)
-    # ---- headline: device-resident inputs, whole step
-    ms_total = timed(step, args.steps)
+    # ---- headline: device-resident inputs, whole step.  Blocks of exactly --steps steps are repeated until MIN_TIMED_MS
+    #      of device time are covered, and the median block is reported (a single block of 20 steps lasts 1 ms).
+    blocks = timed_blocks(step, args.steps, MIN_TIMED_MS, stream, barrier, world, dev)
+    ms_total = statistics.median(blocks)
     # ---- per-kernel: events around every launch of the step's kernel (back to back in the loop above a launch's
     #      set-up overlaps the end of the one before it; here it does not)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    n_iso = max(args.steps, 100)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_iso)]
     barrier()
-    for i in range(args.steps):
+    for i in range(n_iso):
         evs[i][0].record(stream)
         step(i)
         evs[i][1].record(stream)
@@ -286,7 +324,7 @@ def run_ours(args, rank, world, local_rank):
 
     for i in range(3):
         step_host(i)
-    ms_e2e_eager = timed(step_host, args.steps)
+    ms_e2e_eager = statistics.median(timed_blocks(step_host, args.steps, MIN_TIMED_MS / 2, stream, barrier, world, dev))
     same = torch.equal(out_h, out.cpu())
     # The same call captured once per cache copy into a CUDA graph (copy in, one kernel, copy out) and replayed:
     # what a serving loop does with a fixed-shape decode step.  The graph reads the pinned buffers at replay time.
@@ -309,15 +347,7 @@ def run_ours(args, rank, world, local_rank):
             for i in range(3):
                 step_graph(i)
             ok = torch.equal(out_h, out.cpu())
-            barrier()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(side)
-            for i in range(args.steps):
-                step_graph(i)
-            e1.record(side)
-            torch.cuda.synchronize()
-            ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
-            barrier()
+            ms = statistics.median(timed_blocks(step_graph, args.steps, MIN_TIMED_MS / 2, side, barrier, world, dev))
         return ms, ok
 
     ms_e2e = ms_e2e_eager
@@ -326,15 +356,16 @@ def run_ours(args, rank, world, local_rank):
         same = same and same_graph
     clocks = sampler.stop() if sampler else None
 
-    # ---- extra single-GPU context numbers (not part of the headline): prefill of workload 3
+    # ---- the other workloads, single GPU only (context beside the headline, and the numbers the targets are set on)
     extra = {}
     if rank == 0 and world == 1 and not args.no_extra:
         extra = extra_numbers(slim, workloads, dev)
 
     if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
         return
     hbm_peak, bf16_peak, peak_kind = _peaks()
-    tokens = world * B * args.steps
     cache_bytes = sum(kv_len_host) * Hkv * ROW_BYTES
     # whole step: cache read once, Q in, O out, new K/V rows read as bf16 and written as codes + scales
     step_bytes = cache_bytes + 2 * B * Hq * 256 + B * Hkv * (2 * 256 + ROW_BYTES)
@@ -350,6 +381,7 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": whole_job_rate(B, args.steps, world, ms_total), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps,
+        "repeats": len(blocks), "block_ms": {"median": ms_total, "min": min(blocks), "max": max(blocks)},
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s8 (tcgen05 kind::i8 MMA, s32 accumulate; fp32 softmax)",
         "data": "synthetic",
         "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
@@ -362,7 +394,7 @@ def run_ours(args, rank, world, local_rank):
                      "unit": "GB/s", "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_8tbs": achieved / 8000.0, "bytes_per_launch": split_bytes,
                      "avg_launch_ms": split_avg_ms, "isolated_launch_ms": statistics.mean(split_ms),
-                     "isolated_min_launch_ms": min(split_ms), "traffic": TRAFFIC_PER_LAUNCH},
+                     "isolated_min_launch_ms": min(split_ms), "traffic": stored_traffic()},
         "e2e": {"value": whole_job_rate(B, args.steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps, "matches_device_path": bool(same),
                 "launch": ("slim_decode_step_host called and synchronised every step" if args.no_graph else
@@ -375,15 +407,103 @@ def run_ours(args, rank, world, local_rank):
     if world == 1 and not args.no_cpu:
         line["cpu_baseline"] = cpu_baseline(w)
     if extra:
+        line["targets"] = targets_summary(line, extra)
         line["extra"] = extra
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
-# dram bytes read + written by one slim_decode_stream_kernel launch on this workload (281.29 MB read,
-# 5.82 MB written), from the ncu capture summarised under profiles/.
-TRAFFIC_PER_LAUNCH = 286.23e6
+def targets_summary(line, extra):
+    """The figures the targets are set on, side by side: decode attention as a fraction of 8 TB/s (target 0.70) and
+    prefill attention as a fraction of the measured dense bf16 rate (target 0.50); append against the copy rate."""
+    def dec(key):
+        d = extra.get(key)
+        return None if d is None else {"us": 1e3 * d["ms"], "frac_of_8tbs": d["gbs"] / 8000.0, "target": 0.70,
+                                       "met": d["gbs"] / 8000.0 >= 0.70}
+
+    def pre(key):
+        d = extra.get(key)
+        return None if d is None else {"ms": d["ms"], "tflops": d["tflops"], "frac_of_bf16_peak": d["frac_of_bf16_peak"],
+                                       "kernel": "slim_attn_prefill (streamed form)", "target": 0.50,
+                                       "met": d["frac_of_bf16_peak"] >= 0.50}
+    t = {"decode_c2_step": {"us": 1e3 * line["ms_per_step"], "frac_of_8tbs": line["roofline"]["frac_of_8tbs"], "target": 0.70,
+                            "met": line["roofline"]["frac_of_8tbs"] >= 0.70},
+         "decode_c4": dec("decode_c4"), "decode_c4_step": dec("step_c4"),
+         "prefill_c3": pre("prefill_c3"), "prefill_c5": pre("prefill_c5")}
+    if "append_c3" in extra:
+        t["append_c3"] = {"us": 1e3 * extra["append_c3"]["ms"], "frac_of_hbm_peak": extra["append_c3"]["frac_of_hbm_peak"]}
+    return t
+
+
+def run_sharded(args, rank, world, dev, barrier):
+    """--shard: ONE workload's decode attention divided over the ranks (strong scaling): workload 4 by kv heads
+    (64 query heads over 8 kv heads: one kv head per rank at 8 GPUs), workload 5 (2 kv heads) by key ranges with one
+    all-gather of the row partials per step.  Every rank's kernels read its own GPU's memory only."""
+    import torch
+    import torch.distributed as dist
+    from paper_2407_07304_b200 import workloads
+    from paper_2407_07304_b200.shard import ShardPlan, ShardedLayer
+    w = workloads.make_workload(args.shard_workload)
+    lens = [w.total_len(b) - w.decode_steps + 1 for b in range(w.B)]
+    plan = ShardPlan(w.Hq, w.Hkv, lens, world)
+    shard = plan.shard(rank)
+    group = None
+    if plan.parts > 1 and plan.parts < world:
+        # every rank creates every group (torch.distributed's rule); it keeps its own
+        for h in range(w.Hkv):
+            ranks = [h * plan.parts + i for i in range(plan.parts)]
+            g = dist.new_group(ranks)
+            if rank in ranks:
+                group = g
+    copies = max(1, min(12, int(2.5e9 // max(1, plan.cache_bytes(rank)))))   # rotated copies of this rank's cache
+    layers = []
+    for _ in range(copies):
+        layer = ShardedLayer(w, plan, rank, device=dev, group=group)
+        if layers:
+            layer.cache.codes.copy_(layers[0].cache.codes)
+            layer.cache.scales.copy_(layers[0].cache.scales)
+        else:
+            layer.fill()
+        layers.append(layer)
+    q = w.q_decode[0].to(dev).contiguous()
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        layers[i % copies].decode(q, stream)
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    sampler = ClockSampler(dev.index) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.1)
+    blocks = timed_blocks(step, args.steps, MIN_TIMED_MS, stream, barrier, world, dev)
+    clocks = sampler.stop() if sampler else None
+    if rank != 0:
+        return
+    ms_total = statistics.median(blocks)
+    hbm_peak, _, peak_kind = _peaks()
+    total_bytes = sum(lens) * w.Hkv * ROW_BYTES + 2 * w.B * w.Hq * 256
+    achieved = total_bytes / world / (ms_total / args.steps * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": w.B * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_total / args.steps, "repeats": len(blocks),
+        "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+        "dtype": "s8 (tcgen05 kind::i8 MMA, s32 accumulate; fp32 softmax)", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": 128,
+                   "parallelism": (f"tp{world} by kv heads, no collective" if plan.mode == "heads" else
+                                   f"{w.Hkv} kv heads x {plan.parts} key ranges, one all-gather of "
+                                   f"{w.B * len(shard.q_heads) * 528} B per rank and step"),
+                   "l2": f"{copies} copies of each rank's {plan.cache_bytes(rank) / 1e6:.0f} MB cache share rotated"},
+        "roofline": {"bound": "hbm", "kernel": "slim_decode_stream_kernel", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                     "frac": achieved / hbm_peak, "peak_kind": f"of {peak_kind}, per GPU", "traffic": None},
+        "gpu_launches": args.steps * (2 if plan.mode == "heads" else 3), "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+
+
+MIN_TIMED_MS = 200.0       # device time covered by the timed blocks of the headline number
 
 
 def extra_numbers(slim, workloads, dev):
@@ -426,31 +546,39 @@ def extra_numbers(slim, workloads, dev):
     hbm_peak, _, _ = _peaks()
     del run, q, out, k_new, v_new
 
+    def rotated_caches(w, ctx, copies):
+        """`copies` caches filled with the first ctx[b] tokens of every sequence, each in memory of its own."""
+        r = LayerRun(w, device=dev)
+        r.append(ctx)
+        caches = [r.cache]
+        for _ in range(copies - 1):
+            c = slim.SlimCache(w.B, w.Hkv, w.pages_per_seq(), device=dev)
+            c.codes.copy_(r.cache.codes)
+            c.scales.copy_(r.cache.scales)
+            caches.append(c)
+        return r, caches
+
     def decode_numbers(index, copies, label):
         """slim_attn_decode (split + merge) of workload `index` at its final context, cache pre-filled untimed."""
         w = workloads.make_workload(index)
-        runs = []
-        for _ in range(copies):
-            r = LayerRun(w, device=dev)
-            ctx = [w.total_len(b) - w.decode_steps for b in range(w.B)]
-            r.append(ctx)
-            r.append([1] * w.B)
-            runs.append(r)
+        ctx = [w.total_len(b) - w.decode_steps + 1 for b in range(w.B)]
+        r, caches = rotated_caches(w, ctx, copies)
         qd = w.q_decode[0].to(dev).contiguous()
         od = torch.empty_like(qd)
-        kvl = torch.tensor(runs[0].pos, dtype=torch.int32, device=dev)
-        mk = max(runs[0].pos)
+        kvl = torch.tensor(ctx, dtype=torch.int32, device=dev)
+        mk = max(ctx)
         it = [0]
 
         def dec():
-            c = runs[it[0] % copies]
+            c = caches[it[0] % copies]
             it[0] += 1
-            slim.slim_attn_decode(c.cache, qd, od, kvl, w.B, mk, w.Hq, w.sm_scale, runs[0].ws_decode, stream)
+            slim.slim_attn_decode(c, qd, od, kvl, w.B, mk, w.Hq, w.sm_scale, r.ws_decode, stream)
 
-        ms = time_it(dec, 50)
-        nbytes = sum(runs[0].pos) * w.Hkv * ROW_BYTES + 2 * w.B * w.Hq * 256
+        ms = time_it(dec, 10 * copies if copies > 1 else 50)
+        nbytes = sum(ctx) * w.Hkv * ROW_BYTES + 2 * w.B * w.Hq * 256
         return {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
-                "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "cache": label}
+                "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "frac_of_8tbs": nbytes / (ms * 1e-3) / 1e9 / 8000.0,
+                "cache": label}
 
     def prefill_numbers(index, shrink=1, reps=3, two_pass=False):
         w = workloads.make_workload(index, shrink=shrink)
@@ -513,33 +641,41 @@ def extra_numbers(slim, workloads, dev):
         return {"workload": w.name + f"_last{n}", "q_tokens": n, "kv_tokens": S_, "ms": ms,
                 "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_bf16_peak": fl / (ms * 1e-3) / 1e12 / bf16_peak}
 
-    def step_numbers(index, label):
+    def step_numbers(index, label, copies=1):
         """slim_decode_step (append of one token per sequence + decode in one call) at the workload's final context."""
         w = workloads.make_workload(index)
-        r = LayerRun(w, device=dev)
         ctx = [w.total_len(b) - 1 for b in range(w.B)]
-        r.append(ctx)
+        r, caches = rotated_caches(w, ctx, copies)
         kn = torch.stack([r.k[b][ctx[b]] for b in range(w.B)]).contiguous()
         vn = torch.stack([r.v[b][ctx[b]] for b in range(w.B)]).contiguous()
         qd = w.q_decode[0].to(dev).contiguous()
         od = torch.empty_like(qd)
         kvl = torch.tensor([c + 1 for c in ctx], dtype=torch.int32, device=dev)
+        it = [0]
 
         def st():
-            slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, stream)
+            c = caches[it[0] % copies]
+            it[0] += 1
+            slim.slim_decode_step(c, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, stream)
 
-        ms = time_it(st, 50)
+        ms = time_it(st, 10 * copies if copies > 1 else 50)
+        nbytes = (sum(ctx) + w.B) * w.Hkv * ROW_BYTES + 2 * w.B * w.Hq * 256 + w.B * w.Hkv * (2 * 256 + ROW_BYTES)
+        res = {"workload": w.name, "ms": ms, "tokens_per_s": w.B / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
+               "frac_of_8tbs": nbytes / (ms * 1e-3) / 1e9 / 8000.0, "cache": label}
+        if copies > 1:
+            return res
         # the same step replayed from a CUDA graph of twenty calls: the device-side latency of a step without the
         # host's launch cost between steps (the same new row goes to the same slot every time: idempotent)
         side = torch.cuda.Stream()
         n_in_graph = 20
+        c0 = caches[0]
         with torch.cuda.stream(side):
-            slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, side)
+            slim.slim_decode_step(c0, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, side)
             side.synchronize()
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
                 for _ in range(n_in_graph):
-                    slim.slim_decode_step(r.cache, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, side)
+                    slim.slim_decode_step(c0, qd, kn, vn, od, kvl, w.B, max(ctx) + 1, w.Hq, w.sm_scale, r.ws_decode, side)
             g.replay()
             side.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -548,12 +684,13 @@ def extra_numbers(slim, workloads, dev):
                 g.replay()
             e1.record(side)
             side.synchronize()
-            ms_graph = e0.elapsed_time(e1) / (5 * n_in_graph)
-        return {"workload": w.name, "ms": ms, "ms_graph_replay": ms_graph, "tokens_per_s": w.B / (ms * 1e-3), "cache": label}
+            res["ms_graph_replay"] = e0.elapsed_time(e1) / (5 * n_in_graph)
+        return res
 
     more = {}
     if not os.environ.get("SLIM_BENCH_SHORT"):
-        more = {"decode_c4": decode_numbers(4, 2, "two cache copies rotated (2 x 187 MB > L2)"),
+        more = {"decode_c4": decode_numbers(4, 12, "twelve cache copies rotated (12 x 187 MB)"),
+                "step_c4": step_numbers(4, "twelve cache copies rotated (12 x 187 MB)", copies=12),
                 "decode_c5": decode_numbers(5, 1, "17 MB, L2-resident: a latency number, not an HBM number"),
                 "decode_c1": decode_numbers(1, 1, "2 MB, L2-resident: a latency number, not an HBM number"),
                 "prefill_c5": prefill_numbers(5),
@@ -586,6 +723,10 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-extra", action="store_true", help="skip the prefill context numbers")
     ap.add_argument("--no-graph", action="store_true", help="end-to-end leg without CUDA-graph replay (plain calls)")
+    ap.add_argument("--shard", action="store_true",
+                    help="divide ONE workload's decode attention over the ranks (strong scaling) instead of replicating workload 2")
+    ap.add_argument("--shard-workload", type=int, default=4, choices=[2, 4, 5],
+                    help="workload divided by --shard: 4 (by kv heads) or 5 (2 kv heads: by key ranges beyond 2 ranks)")
     ap.add_argument("--extra-only", action="store_true",
                     help="run only the workload-3 prefill/append timings (for profiling that kernel) and print them")
     args = ap.parse_args()
