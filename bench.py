@@ -580,7 +580,7 @@ def extra_numbers(slim, workloads, dev):
                 "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / hbm_peak, "frac_of_8tbs": nbytes / (ms * 1e-3) / 1e9 / 8000.0,
                 "cache": label}
 
-    def prefill_numbers(index, shrink=1, reps=3, two_pass=False):
+    def prefill_numbers(index, shrink=1, reps=3, two_pass=False, full_row=False):
         w = workloads.make_workload(index, shrink=shrink)
         r = LayerRun(w, device=dev)
         n = w.prefill_len[0]
@@ -590,7 +590,7 @@ def extra_numbers(slim, workloads, dev):
         q5 = w.q_prefill[0].to(dev).contiguous()
         o5 = torch.empty_like(q5)
 
-        call = slim.slim_attn_prefill_two_pass if two_pass else slim.slim_attn_prefill
+        call = slim.slim_attn_prefill_full_row if full_row else (slim.slim_attn_prefill_two_pass if two_pass else slim.slim_attn_prefill)
 
         def pf():
             call(r.cache, q5, o5, cu5, kv5, 1, n, n, w.Hq, w.sm_scale, r.ws_prefill, stream)
@@ -700,6 +700,8 @@ def extra_numbers(slim, workloads, dev):
                 # the literal order (all scores of a row, then softmax, then .V): maxima first, no corrections
                 "prefill_two_pass_c3": prefill_numbers(3, two_pass=True),
                 "prefill_two_pass_sweep": [prefill_numbers(3, shrink=k, reps=10, two_pass=True) for k in (32, 16, 8, 4, 2)],
+                # the other literal order: the whole score row of a 128-row block on chip, one softmax (caches up to 256 tokens)
+                "prefill_full_row_256": prefill_numbers(3, shrink=32, reps=10, full_row=True),
                 "prefill_batched": batched_prefill_numbers(),
                 "prefill_chunked": chunked_prefill_numbers(),
                 # one sequence, 32 heads, the sequence lengths of the paper's Table 3 (256 ... 4096 tokens)

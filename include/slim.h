@@ -150,6 +150,26 @@ int slim_attn_prefill_two_pass(const slim_cache_t *cache, const void *q, void *o
                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same attention with the whole score row on chip, the other literal form
+ * of Section 2.1 (and the first row of the paper's Table 3, 256 tokens): for a
+ * block of 128 query rows every score against all its keys is formed into one
+ * strip of tensor memory, each row gets one softmax over its finished scores
+ * (maximum, exponentials, sum - no running maximum, no second sweep over the
+ * keys), and the strip is multiplied by V.  The strip is 128 rows x 256 fp32
+ * scores beside the 128 x 128 output, which is what tensor memory holds: the
+ * call serves caches of at most SLIM_FULL_ROW_MAX_KEYS tokens and returns
+ * SLIM_ERR_UNSUPPORTED (nothing launched) when max_kv is larger; a kv_len[b]
+ * beyond that limit attends over the first SLIM_FULL_ROW_MAX_KEYS tokens.
+ * Arguments, layout, workspace and error behaviour otherwise as for
+ * slim_attn_prefill; the results agree within the output tolerance.
+ */
+#define SLIM_FULL_ROW_MAX_KEYS 256
+int slim_attn_prefill_full_row(const slim_cache_t *cache, const void *q, void *out,
+                               const int32_t *cu_q, const int32_t *kv_len,
+                               int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq, float sm_scale,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Decode attention: one query token per sequence against all kv_len[b] cached
  * tokens (the new token's K/V already appended).  Same arithmetic as above with
  * q_len == 1.  The next-token phase is a matrix-vector product bound by memory

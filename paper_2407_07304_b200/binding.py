@@ -24,7 +24,7 @@ HEAD_DIM = 128
 PAGE_TOKENS = 128
 
 EXPORTS = (
-    "slim_kv_append", "slim_attn_prefill", "slim_attn_prefill_two_pass", "slim_attn_decode", "slim_attn_decode_split",
+    "slim_kv_append", "slim_attn_prefill", "slim_attn_prefill_two_pass", "slim_attn_prefill_full_row", "slim_attn_decode", "slim_attn_decode_split",
     "slim_attn_decode_merge", "slim_attn_decode_static", "slim_static_status", "slim_static_reset",
     "slim_static_selftest_timeout", "slim_attn_decode_partial", "slim_attn_merge_partials", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
@@ -75,6 +75,8 @@ def lib():
         L.slim_attn_prefill.restype = ctypes.c_int
         L.slim_attn_prefill_two_pass.argtypes = [CP, P, P, P, P, I, I, I, I, F, P, Z, P]
         L.slim_attn_prefill_two_pass.restype = ctypes.c_int
+        L.slim_attn_prefill_full_row.argtypes = [CP, P, P, P, P, I, I, I, I, F, P, Z, P]
+        L.slim_attn_prefill_full_row.restype = ctypes.c_int
         L.slim_attn_decode.argtypes = [CP, P, P, P, I, I, I, F, P, Z, P]
         L.slim_attn_decode.restype = ctypes.c_int
         L.slim_attn_decode_split.argtypes = [CP, P, P, P, P, I, I, I, F, P, Z, P]
@@ -182,6 +184,17 @@ def slim_attn_prefill_two_pass(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq
     rc = lib().slim_attn_prefill_two_pass(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(cu_q), _ptr(kv_len),
                                           B, max_q, max_kv, Hq, sm_scale, _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "slim_attn_prefill_two_pass")
+
+
+FULL_ROW_MAX_KEYS = 256
+
+
+def slim_attn_prefill_full_row(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace=None, stream=None):
+    """Prefill with the whole score row on chip (caches of at most FULL_ROW_MAX_KEYS tokens)."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().slim_attn_prefill_full_row(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(cu_q), _ptr(kv_len),
+                                          B, max_q, max_kv, Hq, sm_scale, _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "slim_attn_prefill_full_row")
 
 
 def slim_attn_decode(cache, q, out, kv_len, B, max_kv, Hq, sm_scale, workspace, stream=None):

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libslim.so")
-SOURCES = ["slim_abi.cu", "slim_append.cu", "slim_decode.cu", "slim_decode_stream.cu", "slim_tmap.cu", "slim_prefill_tc.cu"]
+SOURCES = ["slim_abi.cu", "slim_append.cu", "slim_decode.cu", "slim_decode_stream.cu", "slim_tmap.cu", "slim_prefill_tc.cu", "slim_prefill_row.cu"]
 
 
 def _nvcc():

@@ -28,6 +28,8 @@ int launch_merge_partials(const float *parts, int R, int rows, void *out, cudaSt
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                       int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass);
+int launch_prefill_row(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
+                       int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 size_t prefill_workspace_bytes();
 
 static int check_cache(const slim_cache_t *c)
@@ -58,9 +60,11 @@ SLIM_EXPORT int slim_kv_append(const slim_cache_t *cache, const void *k_new, con
     return launch_append(cache, k_new, v_new, cu_new, start_pos, B, max_new, (cudaStream_t)stream);
 }
 
+enum PrefillVariant { kPrefillStreamed, kPrefillTwoPass, kPrefillFullRow };
+
 static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
                          const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
-                         float sm_scale, void *workspace, size_t workspace_bytes, void *stream, bool two_pass)
+                         float sm_scale, void *workspace, size_t workspace_bytes, void *stream, PrefillVariant variant)
 {
     int rc = check_cache(cache);
     if (rc != SLIM_OK) return rc;
@@ -73,21 +77,33 @@ static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, co
     if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
     const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
-    return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream, two_pass);
+    if (variant == kPrefillFullRow) {
+        if (max_kv > SLIM_FULL_ROW_MAX_KEYS) return SLIM_ERR_UNSUPPORTED;   // the score strip of a row block must fit tensor memory
+        return launch_prefill_row(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream);
+    }
+    return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream,
+                             variant == kPrefillTwoPass);
 }
 
 SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
                                   const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
                                   float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
 {
-    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, false);
+    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, kPrefillStreamed);
 }
 
 SLIM_EXPORT int slim_attn_prefill_two_pass(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
                                            const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
                                            float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
 {
-    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, true);
+    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, kPrefillTwoPass);
+}
+
+SLIM_EXPORT int slim_attn_prefill_full_row(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
+                                           const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
+                                           float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return prefill_entry(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace, workspace_bytes, stream, kPrefillFullRow);
 }
 
 // Shared validation of the decode entry points; *launch is false for a valid no-op.

@@ -44,9 +44,10 @@ class LayerRun:
             self.pos[b] += counts[b]
 
     # ------------------------------------------------------------------ attention
-    def prefill(self, q_list, two_pass=False):
+    def prefill(self, q_list, two_pass=False, full_row=False):
         """Causal attention of q_list[b] (bf16 [n_b, Hq, 128], the last n_b cached positions);
-        two_pass selects slim_attn_prefill_two_pass (maxima first, then P.V, no corrections)."""
+        two_pass selects slim_attn_prefill_two_pass (maxima first, then P.V, no corrections), full_row
+        slim_attn_prefill_full_row (the whole score row on chip; caches of at most 256 tokens)."""
         w = self.w
         lens = [int(q.shape[0]) for q in q_list]
         q = torch.cat([t.to(self.device) for t in q_list]).contiguous()
@@ -54,7 +55,7 @@ class LayerRun:
         cu = [0]
         for n in lens:
             cu.append(cu[-1] + n)
-        fn = slim.slim_attn_prefill_two_pass if two_pass else slim.slim_attn_prefill
+        fn = slim.slim_attn_prefill_full_row if full_row else (slim.slim_attn_prefill_two_pass if two_pass else slim.slim_attn_prefill)
         fn(self.cache, q, out, self._i32(cu), self._i32(self.pos), w.B, max(lens), max(self.pos), w.Hq, w.sm_scale,
            self.ws_prefill)
         return [out[cu[b]:cu[b + 1]] for b in range(w.B)]

@@ -193,6 +193,72 @@ def test_two_pass_prefill_c3_full_sampled_rows():
     _check_two_pass(workloads.make_workload(3), prefill_rows=24)
 
 
+def _check_full_row(w, tails=None, row_relative=False):
+    """slim_attn_prefill_full_row (all scores of a row block on chip, one softmax, then .V) against the oracle;
+    row_relative: error relative to each row's largest output (for inputs whose outputs span many binades)."""
+    from paper_2407_07304_b200 import binding as slim, harness
+    oc = _oracle_cache(w)
+    run = harness.LayerRun(w)
+    run.append(w.prefill_len)
+    qs = w.q_prefill if tails is None else [w.q_prefill[b][w.prefill_len[b] - tails[b]:] for b in range(w.B)]
+    out = run.prefill(qs, full_row=True)
+    ref = run.prefill(qs)
+    torch.cuda.synchronize()
+    assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
+    for b in range(w.B):
+        n = w.prefill_len[b]
+        sel = None if tails is None else list(range(n - tails[b], n))
+        want = so.attention(bf16_bits(w.q_prefill[b]), *oc[b], n, w.sm_scale, sel=sel)
+        if row_relative:
+            got = out[b].float().cpu().numpy().astype(np.float64)
+            denom = np.maximum(np.abs(want).max(axis=-1, keepdims=True), 1e-30)
+            assert np.isfinite(got).all() and (np.abs(got - want) / denom).max() < 2e-2
+            continue
+        _assert_close(out[b], want, f"{w.name} full-row prefill seq {b}")
+        if n > 0:
+            d = (out[b].float() - ref[b].float()).abs().max().item()
+            assert d <= 2 * MAX_ABS, f"{w.name} seq {b}: full-row and streamed outputs differ by {d}"
+
+
+def test_full_row_prefill_c1_all_outputs():
+    _check_full_row(workloads.make_workload(1))       # 256 tokens, 32 heads: every output
+
+
+@pytest.mark.parametrize("lens", [[1], [2, 127], [128, 129], [255, 256, 31], [200, 1, 64, 130]])
+def test_full_row_prefill_ragged_lengths(lens):
+    B = len(lens)
+    _check_full_row(_custom(B, 4, 2, lens, [0] * B, 0, 1700 + lens[0]))
+
+
+def test_full_row_prefill_every_length_to_256():
+    # every prompt length from 1 to 256 in batches of sixteen sequences, grouped-query heads (3 query heads per kv head)
+    for first in range(1, 257, 16):
+        lens = list(range(first, first + 16))
+        _check_full_row(_custom(16, 3, 1, lens, [0] * 16, 0, 1800 + first))
+
+
+def test_full_row_prefill_with_cached_prefix_and_scale_jump():
+    # q_len < kv_len: the last 70 of 250 cached tokens attend ...
+    _check_full_row(_custom(1, 8, 2, [250], [0], 0, 1900), tails=[70])
+    # ... and with the second key tile's K 2^12 smaller and its V 2^9 larger than the first one's (each key tile is
+    # normalised by its own power of two); the outputs span many binades, so the error is taken relative to the row
+    w = _custom(1, 8, 2, [250], [0], 0, 1901)
+    w.k[0][128:] *= 2.0 ** -12
+    w.v[0][128:] *= 2.0 ** 9
+    _check_full_row(w, tails=[70], row_relative=True)
+
+
+def test_full_row_prefill_rejects_longer_caches():
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = _custom(1, 2, 1, [300], [0], 0, 1950)
+    run = harness.LayerRun(w)
+    run.append([300])
+    with pytest.raises(slim.SlimError) as e:
+        run.prefill(w.q_prefill, full_row=True)
+    assert e.value.code == slim.SLIM_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+
+
 def test_c5_full_sampled():
     _check(workloads.make_workload(5), prefill_rows=24, decode_steps={0, 31, 63})
 
