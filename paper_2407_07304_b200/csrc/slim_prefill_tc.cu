@@ -8,10 +8,14 @@
 // while the softmax of one query tile runs on the ALUs the tensor cores work for the other one.
 //
 //   warp 12     loader: TMA tensor copies of the raw INT8 K / V tiles (128-byte swizzle) and bulk copies
-//               of their scales into a 5-stage ring, completion counted on mbarriers
-//   warps 8-11  dequantise in registers (the hybrid-dtype step of Section 2.2): INT8 codes -> fp16
-//               code * scale / 2^e, written in the swizzled layout the tensor cores read (one K and
-//               one V operand buffer; a buffer is refilled as soon as the MMAs that read it are done)
+//               of their scales into one raw stage for K tiles and one for V tiles, completion counted on
+//               mbarriers; the tiles of the next step are prefetched into the L2 a step ahead
+//   warps 8-11, 14, 15  dequantise in registers (the hybrid-dtype step of Section 2.2): INT8 codes -> fp16
+//               code * scale / 2^e, written in the swizzled layout the tensor cores read.  Two K and two V
+//               operand buffers: the converters run a key tile ahead of the tensor cores (with one buffer each
+//               the conversion of V(j) and K(j+1) sat between P.V(j-1) and Q.K(j+1)^T on the critical path).
+//               A thread of warps 8-11 owns a token row and converts six of its eight 16-code pieces, the
+//               two spare warps of the last warp group take the other two pieces of every row
 //   warp 13     one thread issues tcgen05.mma in the order  P0.V(j), Q0.K(j+1)^T, P1.V(j), Q1.K(j+1)^T:
 //               S_t = Q_t . K^T (both operands in shared memory), O_t += P_t . V (P read from tensor
 //               memory), fp32 accumulators in tensor memory
@@ -36,26 +40,25 @@ namespace slim {
 constexpr int kPfThreads = 512;   // four warp groups: softmax 0, softmax 1, dequantisers, {loader, MMA thread, two idle warps}
 constexpr int kPfBM = 128, kPfBN = 128;
 constexpr int kPfRows = 2 * kPfBM;             // query rows per block
-constexpr int kPfRawStages = 5;
+constexpr int kPfRawStages = 2;                // one raw stage for K tiles, one for V tiles
+constexpr int kPfConvWarps = 6;                // warps 8-11 and the two spare warps of the last warp group
 constexpr uint32_t kPfTmemCols = 512;
 constexpr uint32_t kPfTmemS = 0, kPfTmemO = 256;   // S_t at columns 128 t, O_t at 256 + 128 t
 constexpr float kPfRescaleThreshold = 8.f;     // log2 units
 
 namespace pfl {   // shared-memory map
 constexpr uint32_t kQ = 0;                      // two fp16 Q tiles; a tile = two 64-dim halves of [128 rows][128 B]
-constexpr uint32_t kKf = 65536;                 // fp16 K tile, same layout
-constexpr uint32_t kVf = kKf + 32768;           // fp16 V tile: two 64-dim halves of [128 keys][128 B]
-constexpr uint32_t kRaw = kVf + 32768;          // raw stages: 16 KB INT8 tile + 512 B scales (+ pad)
-constexpr uint32_t kRawStage = 17408;
-constexpr uint32_t kMisc = kRaw + kPfRawStages * kRawStage;
+constexpr uint32_t kKf = 65536;                 // two fp16 K tiles (key tiles j even / odd), same layout
+constexpr uint32_t kVf = kKf + 2 * 32768;       // two fp16 V tiles: two 64-dim halves of [128 keys][128 B] each
+constexpr uint32_t kRaw = kVf + 2 * 32768;      // raw INT8 tiles: stage 0 K, stage 1 V (16 KB each, 1 KB aligned for the swizzle)
+constexpr uint32_t kRawScales = kRaw + kPfRawStages * 16384;   // their scales, 512 B per stage
+constexpr uint32_t kMisc = kRawScales + kPfRawStages * 512;
 constexpr uint32_t kRowScale = kMisc + 512;     // float[2][128]: row scale of every query row (written by the thread that converts the row)
 constexpr uint32_t kBytes = kRowScale + 1024;
-// kMisc: floats by parity of the key tile j: [0,2) kexp, [2,4) log2 vexp, [12,14) 1 / vexp; converter warp maxima
-//        [4,12) for K tiles and [20,28) for V tiles; byte 64: tensor-memory address; byte 72: failure flag;
-//        byte 128..: mbarriers
-enum Bar { RAW_FULL = 0, RAW_EMPTY = kPfRawStages, KF_FULL = 2 * kPfRawStages, KF_EMPTY, VF_FULL, VF_EMPTY,
-           S_FULL, P_FULL = S_FULL + 2, O_DONE = P_FULL + 2, Q_FULL = O_DONE + 2, VEXP_FULL = Q_FULL + 2,
-           NUM_BARS = VEXP_FULL + 2 };
+// kMisc: floats by the key tile's position j mod 4: [0,4) kexp, [4,8) log2 vexp, [8,12) 1 / vexp;
+//        byte 64: tensor-memory address; byte 72: failure flag; byte 128..: mbarriers
+enum Bar { RAW_FULL = 0, RAW_EMPTY = 2, KF_FULL = 4, KF_EMPTY = 6, VF_FULL = 8, VF_EMPTY = 10,
+           S_FULL = 12, P_FULL = 14, O_DONE = 16, Q_FULL = 18, VEXP_FULL = 20, NUM_BARS = 24 };
 static_assert(128 + 8 * NUM_BARS <= 512, "mbarriers fit the misc area");
 static_assert(kBytes <= 232448, "shared memory budget of one block");
 }  // namespace pfl
@@ -169,16 +172,20 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     int page_next = 0;
     auto request_raw = [&](int i) {
         const int32_t *bt = p.block_table + (size_t)b * p.max_pages_per_seq;
-        const int slot = i % kPfRawStages, j = i >> 1;
-        const int kv = i & 1;
+        const int kv = i & 1, j = i >> 1;   // K tiles go through raw stage 0, V tiles through stage 1
         int page = page_next;
-        if (kv == 1 && j + 1 < NT) page_next = __ldg(bt + ((kTwoPass && j + 1 >= T) ? j + 1 - T : j + 1));   // requested one tile ahead
         page = (page >= 0 && page < p.num_pages) ? page : 0;
-        const uint32_t dst = sbase + pfl::kRaw + slot * pfl::kRawStage;
-        const uint32_t full = bar(pfl::RAW_FULL, slot);
+        const uint32_t full = bar(pfl::RAW_FULL, kv);
         tc::mbar_arrive_expect_tx(full, 16384 + 512);
-        tc::tma_load_2d(dst, &codes_map, 0, ((page * p.Hkv + head) * 2 + kv) * kPageTokens, full);
-        tc::bulk_load(dst + 16384, p.scales + scale_block_offset(page, head, kv, p.Hkv), 512, full);
+        tc::tma_load_2d(sbase + pfl::kRaw + kv * 16384, &codes_map, 0, ((page * p.Hkv + head) * 2 + kv) * kPageTokens, full);
+        tc::bulk_load(sbase + pfl::kRawScales + kv * 512, p.scales + scale_block_offset(page, head, kv, p.Hkv), 512, full);
+        if (kv == 1 && j + 1 < NT) {
+            // the next key tile's page id, and its two tiles on their way into the L2 a step before they are asked for
+            page_next = __ldg(bt + ((kTwoPass && j + 1 >= T) ? j + 1 - T : j + 1));
+            const int pn = (page_next >= 0 && page_next < p.num_pages) ? page_next : 0;
+            tc::tma_prefetch_2d(&codes_map, 0, ((pn * p.Hkv + head) * 2) * kPageTokens);
+            tc::tma_prefetch_2d(&codes_map, 0, ((pn * p.Hkv + head) * 2 + 1) * kPageTokens);
+        }
         ++raw_issued;
     };
     if (warp == 12 && lane == 0) {
@@ -208,18 +215,18 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     }
 
     if (tid == 0) {
-        for (int i = 0; i < kPfRawStages; ++i) tc::mbar_init(bar(pfl::RAW_EMPTY, i), 128);
-        tc::mbar_init(bar(pfl::KF_FULL, 0), 128);
-        tc::mbar_init(bar(pfl::KF_EMPTY, 0), 1);
-        tc::mbar_init(bar(pfl::VF_FULL, 0), 128);
-        tc::mbar_init(bar(pfl::VF_EMPTY, 0), 1);
         for (int t = 0; t < 2; ++t) {
+            tc::mbar_init(bar(pfl::RAW_EMPTY, t), kPfConvWarps);   // (one arrival per converter warp)
+            tc::mbar_init(bar(pfl::KF_FULL, t), kPfConvWarps);
+            tc::mbar_init(bar(pfl::KF_EMPTY, t), 1);
+            tc::mbar_init(bar(pfl::VF_FULL, t), kPfConvWarps);
+            tc::mbar_init(bar(pfl::VF_EMPTY, t), 1);
             tc::mbar_init(bar(pfl::S_FULL, t), 1);
             tc::mbar_init(bar(pfl::P_FULL, t), 128);
             tc::mbar_init(bar(pfl::O_DONE, t), 1);
             tc::mbar_init(bar(pfl::Q_FULL, t), 128);
-            tc::mbar_init(bar(pfl::VEXP_FULL, t), 128);
         }
+        for (int i = 0; i < 4; ++i) tc::mbar_init(bar(pfl::VEXP_FULL, i), 1);
         tc::mbar_init_fence();
         *fail = 0;
     }
@@ -302,10 +309,10 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             wait(bar(pfl::S_FULL, t), (uint32_t)jj & 1u);
             __syncwarp();   // the wait loop may leave the lanes diverged; the tensor-memory ops below are warp-aligned
             tc::fence_after_sync();
-            wait(bar(pfl::VEXP_FULL, jv & 1), (uint32_t)(jv >> 1) & 1u);   // published long before, as a rule
-            const float c = fmaxf(rs * misc_f[jv & 1], 1e-37f);   // row scale * kexp of this key tile (> 0)
-            const float F = misc_f[2 + (jv & 1)];                 // log2 vexp
-            const float vinv = misc_f[12 + (jv & 1)];             // 1 / vexp
+            wait(bar(pfl::VEXP_FULL, jv & 3), (uint32_t)(jv >> 2) & 1u);   // published long before, as a rule
+            const float c = fmaxf(rs * misc_f[jv & 3], 1e-37f);   // row scale * kexp of this key tile (> 0)
+            const float F = misc_f[4 + (jv & 3)];                 // log2 vexp
+            const float vinv = misc_f[8 + (jv & 3)];              // 1 / vexp
             const int key0 = j * kPfBN;
             const bool diag = key0 + kPfBN - 1 > last_key;       // some of this tile's keys are masked for this row
             // ---- the whole score row into registers with one round trip to tensor memory, then its maximum
@@ -436,80 +443,99 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
 #pragma unroll
             for (int i = 0; i < 16; ++i) dst[i] = make_uint4(0, 0, 0, 0);
         }
-    } else if (warp < 12) {
-        // =========================================================== dequantise: thread = token row of the tile
-        const int r = tid - 256, cw = warp - 8;
+    } else if (warp < 12 || warp >= 14) {
+        // =========================================================== dequantise
+        // A thread of warps 8-11 owns token row r = tid - 256 of every tile and converts its pieces 0..5 (a piece =
+        // 16 codes); a thread of warps 14, 15 owns rows 2 u, 2 u + 1 (u = tid - 448) and converts their pieces 6, 7.
+        const bool main_cv = warp < 12;
+        const int r0 = main_cv ? tid - 256 : 2 * (tid - 448);
+        const int n_rows = main_cv ? 1 : 2, c_first = main_cv ? 0 : 6, c_last = main_cv ? 6 : 8;
+        const bool announces = warp == 8 && lane == 0;   // the thread that publishes a tile's exponents
         for (int i = 0; i < 2 * NT; ++i) {
-            const int slot = i % kPfRawStages, j = i >> 1;   // j: position in the block's tile sequence
-            const bool is_k = (i & 1) == 0;   // K tile first, then the V tile of the same keys
-            wait(bar(pfl::RAW_FULL, slot), (uint32_t)(i / kPfRawStages) & 1u);
-            if (is_k) wait(bar(pfl::KF_EMPTY, 0), ((uint32_t)j & 1u) ^ 1u);
-            const unsigned char *raw = smem + pfl::kRaw + slot * pfl::kRawStage;
+            const int kv = i & 1, j = i >> 1;   // j: position in the block's tile sequence; K tile first, then the V tile of the same keys
+            const bool is_k = kv == 0;
+            const int buf = j & 1;
+            wait(bar(pfl::RAW_FULL, kv), (uint32_t)j & 1u);
+            const unsigned char *raw = smem + pfl::kRaw + kv * 16384;
+            const float *scales = reinterpret_cast<const float *>(smem + pfl::kRawScales + kv * 512);
             const int n_valid = min(kPfBN, kvl - ((kTwoPass && j >= T) ? j - T : j) * kPfBN);   // rows past the cache length hold anything: zeroed
-            const float sc = (r < n_valid) ? reinterpret_cast<const float *>(raw + 16384)[r] : 0.f;
-            // power of two below the tile's largest scale; the exchange buffers alternate with j so that a fast
-            // warp cannot overwrite what a slow one still reads
-            float *cm = misc_f + (is_k ? 4 : 20) + 4 * (j & 1);
-            const float wm = warp_max(sc);
-            if (lane == 0) cm[cw] = wm;
-            tc::named_barrier(1, 128);
-            const float tm = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
-            const float ex = (tm > 0.f) ? pow2_floor(tm) : 1.f;
+            // power of two below the tile's largest scale (every warp finds it for itself: four scales per lane)
+            float wm = 0.f;
+            {
+                const float4 s4 = *reinterpret_cast<const float4 *>(scales + 4 * lane);
+                const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (4 * lane + k < n_valid) wm = fmaxf(wm, sv[k]);
+                wm = warp_max(wm);
+            }
+            const float ex = (wm > 0.f) ? pow2_floor(wm) : 1.f;
+            const float rex = pow2_recip(ex);
             if (is_k) {
-                if (r == 0) misc_f[j & 1] = ex;
+                if (announces) misc_f[j & 3] = ex;
+                wait(bar(pfl::KF_EMPTY, buf), ((uint32_t)(j >> 1) & 1u) ^ 1u);
             } else {
                 // the softmax of this key tile needs the V exponent before the V tile itself is converted
-                if (r == 0) {
-                    misc_f[2 + (j & 1)] = (float)((int)(__float_as_uint(ex) >> 23) - 127);   // log2 of the power of two
-                    misc_f[12 + (j & 1)] = pow2_recip(ex);
+                if (announces) {
+                    misc_f[4 + (j & 3)] = (float)((int)(__float_as_uint(ex) >> 23) - 127);   // log2 of the power of two
+                    misc_f[8 + (j & 3)] = rex;
+                    tc::mbar_arrive(bar(pfl::VEXP_FULL, j & 3));
                 }
-                tc::mbar_arrive(bar(pfl::VEXP_FULL, j & 1));
-                wait(bar(pfl::VF_EMPTY, 0), ((uint32_t)j & 1u) ^ 1u);
+                wait(bar(pfl::VF_EMPTY, buf), ((uint32_t)(j >> 1) & 1u) ^ 1u);
             }
-            const float f = sc * pow2_recip(ex);   // scale / 2^e in [0, 2)
-            const uint32_t fac2 = pack_half2(f, f);
-            unsigned char *dstb = smem + (is_k ? pfl::kKf : pfl::kVf) + r * 128;
+            unsigned char *dst_tile = smem + (is_k ? pfl::kKf : pfl::kVf) + buf * 32768;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint4 w4 = *reinterpret_cast<const uint4 *>(raw + r * 128 + ((c ^ (r & 7)) << 4));
-                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-                uint32_t hh[8];
+            for (int q = 0; q < 2; ++q) {
+                if (q >= n_rows) break;
+                const int r = r0 + q;
+                const float f = ((r < n_valid) ? scales[r] : 0.f) * rex;   // scale / 2^e in [0, 2)
+                const uint32_t fac2 = pack_half2(f, f);
+                unsigned char *dstb = dst_tile + r * 128;
+                for (int c = c_first; c < c_last; ++c) {
+                    const uint4 w4 = *reinterpret_cast<const uint4 *>(raw + r * 128 + ((c ^ (r & 7)) << 4));
+                    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+                    uint32_t hh[8];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    // byte u = code ^ 0x80 under 0x64 is the fp16 number 1152 + code
-                    const uint32_t x = w[k] ^ 0x80808080u;
-                    hh[2 * k] = pf_hmul2(pf_hsub2(__byte_perm(x, 0x64646464u, 0x4140), 0x64806480u), fac2);
-                    hh[2 * k + 1] = pf_hmul2(pf_hsub2(__byte_perm(x, 0x64646464u, 0x4342), 0x64806480u), fac2);
+                    for (int k = 0; k < 4; ++k) {
+                        // byte u = code ^ 0x80 under 0x64 is the fp16 number 1152 + code
+                        const uint32_t x = w[k] ^ 0x80808080u;
+                        hh[2 * k] = pf_hmul2(pf_hsub2(__byte_perm(x, 0x64646464u, 0x4140), 0x64806480u), fac2);
+                        hh[2 * k + 1] = pf_hmul2(pf_hsub2(__byte_perm(x, 0x64646464u, 0x4342), 0x64806480u), fac2);
+                    }
+                    const uint32_t hf = (uint32_t)(c >> 2) * 16384u;
+                    const int oc = 2 * (c & 3);
+                    *reinterpret_cast<uint4 *>(dstb + hf + ((oc ^ (r & 7)) << 4)) = make_uint4(hh[0], hh[1], hh[2], hh[3]);
+                    *reinterpret_cast<uint4 *>(dstb + hf + (((oc + 1) ^ (r & 7)) << 4)) = make_uint4(hh[4], hh[5], hh[6], hh[7]);
                 }
-                const uint32_t hf = (uint32_t)(c >> 2) * 16384u;
-                const int oc = 2 * (c & 3);
-                *reinterpret_cast<uint4 *>(dstb + hf + ((oc ^ (r & 7)) << 4)) = make_uint4(hh[0], hh[1], hh[2], hh[3]);
-                *reinterpret_cast<uint4 *>(dstb + hf + (((oc + 1) ^ (r & 7)) << 4)) = make_uint4(hh[4], hh[5], hh[6], hh[7]);
             }
             tc::fence_proxy_async();
-            tc::mbar_arrive(bar(is_k ? pfl::KF_FULL : pfl::VF_FULL, 0));
-            tc::mbar_arrive(bar(pfl::RAW_EMPTY, slot));
+            __syncwarp();
+            if (lane == 0) {
+                tc::mbar_arrive(bar(is_k ? pfl::KF_FULL : pfl::VF_FULL, buf));
+                tc::mbar_arrive(bar(pfl::RAW_EMPTY, kv));
+            }
         }
     } else if (warp == 12) {
         // =========================================================== loader (one thread)
         if (lane == 0 && T > 0) {
-            for (int i = kPfRawStages; i < 2 * NT; ++i) {   // the first round of the ring was requested during set-up
-                wait(bar(pfl::RAW_EMPTY, i % kPfRawStages), ((uint32_t)(i / kPfRawStages) & 1u) ^ 1u);
+            for (int i = kPfRawStages; i < 2 * NT; ++i) {   // the first K and V tile were requested during set-up
+                wait(bar(pfl::RAW_EMPTY, i & 1), ((uint32_t)(i >> 1) & 1u) ^ 1u);
                 request_raw(i);
             }
         }
     } else if (warp == 13) {
-        // =========================================================== MMA issue (one thread); warps 14, 15 only fill the warp group
+        // =========================================================== MMA issue (one thread)
         if (lane == 0 && T > 0) {
             constexpr uint32_t idesc_qk = tc::instr_desc(1, 0, 0, false, false, 128, 128);   // f32 <- f16 x f16, both K-major
             constexpr uint32_t idesc_pv = tc::instr_desc(1, 0, 0, false, true, 128, 128);    // B (V) is MN-major
             // Operand descriptors are built once; an MMA step only adds a constant to the address field.
             const uint64_t dq0 = tc::smem_desc(sbase + pfl::kQ, 16, 1024, tc::kSwizzle128B);
             const uint64_t dq1 = tc::smem_desc(sbase + pfl::kQ + 32768u, 16, 1024, tc::kSwizzle128B);
-            const uint64_t dk = tc::smem_desc(sbase + pfl::kKf, 16, 1024, tc::kSwizzle128B);
-            const uint64_t dv = tc::smem_desc(sbase + pfl::kVf, 16384, 1024, tc::kSwizzle128B);
-            auto issue_qk = [&](int t) {   // S_t = Q_t . K^T
+            const uint64_t dk0 = tc::smem_desc(sbase + pfl::kKf, 16, 1024, tc::kSwizzle128B);      // K^ buffer 0; buffer 1 lies 32 KB behind it
+            const uint64_t dv0 = tc::smem_desc(sbase + pfl::kVf, 16384, 1024, tc::kSwizzle128B);
+            auto issue_qk = [&](int t, int buf) {   // S_t = Q_t . K^T
                 const uint64_t dq = t ? dq1 : dq0;
+                const uint64_t dk = dk0 + (uint64_t)(buf * (32768 >> 4));
                 const uint32_t d = tmem + kPfTmemS + (uint32_t)t * 128u;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -519,8 +545,9 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
                 }
                 tc::commit(bar(pfl::S_FULL, t));
             };
-            auto issue_pv = [&](int t, bool first) {   // O_t (+)= P_t . V
+            auto issue_pv = [&](int t, bool first, int buf) {   // O_t (+)= P_t . V
                 const uint32_t d = tmem + kPfTmemO + (uint32_t)t * 128u, a = tmem + kPfTmemS + (uint32_t)t * 128u;
+                const uint64_t dv = dv0 + (uint64_t)(buf * (32768 >> 4));
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)   // keys [16 ks, 16 ks + 16): 2 KB further down the V tile, 8 columns of P
                     tc::mma_f16_ts(d, a + ks * 8, dv + (uint64_t)((ks * 2048) >> 4), idesc_pv, !first || ks > 0);
@@ -530,44 +557,46 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
             if (T1 > 0) wait(bar(pfl::Q_FULL, 1), 0);
             wait(bar(pfl::KF_FULL, 0), 0);
             tc::fence_after_sync();
-            if (T0 > 0) issue_qk(0);
-            if (T1 > 0) issue_qk(1);
+            if (T0 > 0) issue_qk(0, 0);
+            if (T1 > 0) issue_qk(1, 0);
             tc::commit(bar(pfl::KF_EMPTY, 0));
             // The fixed order P0.V(j), Q0.K(j+1)^T, P1.V(j), Q1.K(j+1)^T keeps the two query tiles half a step
             // apart, so that their softmax phases (which share the special-function units) alternate.
             int c0 = 0, c1 = 0;   // two-pass form: steps each query tile has taken (its barrier phases)
             for (int jv = 0; jv < NT; ++jv) {
-                const uint32_t ph = (uint32_t)jv & 1u, phn = ph ^ 1u;
+                const uint32_t ph = (uint32_t)jv & 1u;                       // parity of the query tiles' barriers at this position
+                const int buf = jv & 1, bufn = buf ^ 1;                      // operand buffers of this position's V tile / the next one's K tile
+                const uint32_t bph = (uint32_t)(jv >> 1) & 1u, bphn = (uint32_t)((jv + 1) >> 1) & 1u;   // parities of those buffers' barriers
                 const bool second = kTwoPass && jv >= T;
                 const int j = second ? jv - T : jv;                          // key tile at this position
                 const int jn = (kTwoPass && jv + 1 >= T) ? jv + 1 - T : jv + 1;   // key tile at the next position
                 const bool more = jv + 1 < NT;
                 const bool a0 = j < T0, a1 = j < T1, n0 = more && jn < T0, n1 = more && jn < T1;
                 const bool pv = !kTwoPass || second;                         // the first pass has no P.V
-                wait(bar(pfl::VF_FULL, 0), ph);
+                wait(bar(pfl::VF_FULL, buf), bph);
                 if (a0) {
                     wait(bar(pfl::P_FULL, 0), kTwoPass ? ((uint32_t)c0 & 1u) : ph);
                     tc::fence_after_sync();
-                    if (pv) issue_pv(0, j == 0); else tc::commit(bar(pfl::O_DONE, 0));
+                    if (pv) issue_pv(0, j == 0, buf); else tc::commit(bar(pfl::O_DONE, 0));
                     ++c0;
                 }
-                if (n0 || n1) wait(bar(pfl::KF_FULL, 0), phn);
+                if (n0 || n1) wait(bar(pfl::KF_FULL, bufn), bphn);
                 if (n0) {
                     tc::fence_after_sync();
-                    issue_qk(0);
+                    issue_qk(0, bufn);
                 }
                 if (a1) {
                     wait(bar(pfl::P_FULL, 1), kTwoPass ? ((uint32_t)c1 & 1u) : ph);
                     tc::fence_after_sync();
-                    if (pv) issue_pv(1, j == 0); else tc::commit(bar(pfl::O_DONE, 1));
+                    if (pv) issue_pv(1, j == 0, buf); else tc::commit(bar(pfl::O_DONE, 1));
                     ++c1;
                 }
-                tc::commit(bar(pfl::VF_EMPTY, 0));
+                tc::commit(bar(pfl::VF_EMPTY, buf));
                 if (n1) {
                     tc::fence_after_sync();
-                    issue_qk(1);
+                    issue_qk(1, bufn);
                 }
-                if (n0 || n1) tc::commit(bar(pfl::KF_EMPTY, 0));
+                if (n0 || n1) tc::commit(bar(pfl::KF_EMPTY, bufn));
             }
         }
     }
@@ -577,7 +606,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     if (warp == 12 && lane == 0 && *fail != 0) {
         // a wait ran out somewhere: give the copies still in flight a bounded chance to land before the block exits
         for (int i = max(0, raw_issued - kPfRawStages); i < raw_issued; ++i)
-            tc::mbar_wait(bar(pfl::RAW_FULL, i % kPfRawStages), (uint32_t)(i / kPfRawStages) & 1u, 1u << 14);
+            tc::mbar_wait(bar(pfl::RAW_FULL, i & 1), (uint32_t)(i >> 1) & 1u, 1u << 14);
         if (p.status != nullptr) atomicExch(p.status, SLIM_ERR_TIMEOUT);
     }
     if (warp == 13) {

@@ -177,6 +177,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void *tmap,
         "l"(tmap), "r"(x), "r"(y), "r"(mbar_smem)
         : "memory");
 }
+// Brings the box at (x, y) of a tiled tensor into the L2 without copying it anywhere (same alignment rule for x).
+__device__ __forceinline__ void tma_prefetch_2d(const void *tmap, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];\n" ::"l"(tmap), "r"(x), "r"(y) : "memory");
+}
 // Asks the copy engine to fetch a tensor map (a kernel parameter) ahead of its first use.
 __device__ __forceinline__ void prefetch_tensormap(const void *tmap)
 {
