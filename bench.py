@@ -259,15 +259,16 @@ def run_ours(args, rank, world, local_rank):
             dist.destroy_process_group()
         return
 
+    n_rot = max(1, args.copies)
     w = workloads.make_workload(2)
     B, Hq, Hkv, ctx = w.B, w.Hq, w.Hkv, w.bulk_len[0]
     kv_len_host = [ctx + 1] * B
 
-    # N_ROT independent caches, each pre-filled (untimed) with the 2048-token context
+    # n_rot independent caches, each pre-filled (untimed) with the 2048-token context
     first = LayerRun(w, device=dev)
     first.append(w.bulk_len)
     runs = [first]
-    for _ in range(N_ROT - 1):
+    for _ in range(n_rot - 1):
         c = slim.SlimCache(B, Hkv, w.pages_per_seq(), device=dev)      # a copy of the filled cache in memory of its own
         c.codes.copy_(first.cache.codes)
         c.scales.copy_(first.cache.scales)
@@ -285,7 +286,7 @@ def run_ours(args, rank, world, local_rank):
     def step(i):
         # one call, one kernel: it quantises the new token's K/V rows into the cache, attends over them from registers,
         # streams the rest of the cache once and merges its own partial results as its blocks finish
-        slim.slim_decode_step(runs[i % N_ROT].cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
+        slim.slim_decode_step(runs[i % n_rot].cache, q, k_new, v_new, out, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
 
     for i in range(max(3, args.warmup)):
         step(i)
@@ -295,7 +296,7 @@ def run_ours(args, rank, world, local_rank):
         time.sleep(0.1)
     # ---- headline: device-resident inputs, whole step.  Blocks of exactly --steps steps are repeated until MIN_TIMED_MS
     #      of device time are covered, and the median block is reported (a single block of 20 steps lasts 1 ms).
-    blocks = timed_blocks(step, args.steps, MIN_TIMED_MS, stream, barrier, world, dev)
+    blocks = timed_blocks(step, args.steps, args.min_ms, stream, barrier, world, dev)
     ms_total = statistics.median(blocks)
     # ---- per-kernel: events around every launch of the step's kernel (back to back in the loop above a launch's
     #      set-up overlaps the end of the one before it; here it does not)
@@ -318,13 +319,13 @@ def run_ours(args, rank, world, local_rank):
     staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
 
     def step_host(i):
-        c = runs[i % N_ROT].cache
+        c = runs[i % n_rot].cache
         slim.slim_decode_step_host(c, q_h, k_h, v_h, out_h, staging, kv_len, B, max_kv, Hq, w.sm_scale, ws, stream)
         stream.synchronize()        # the caller needs the result before the next token
 
     for i in range(3):
         step_host(i)
-    ms_e2e_eager = statistics.median(timed_blocks(step_host, args.steps, MIN_TIMED_MS / 2, stream, barrier, world, dev))
+    ms_e2e_eager = statistics.median(timed_blocks(step_host, args.steps, args.min_ms / 2, stream, barrier, world, dev))
     same = torch.equal(out_h, out.cpu())
     # The same call captured once per cache copy into a CUDA graph (copy in, one kernel, copy out) and replayed:
     # what a serving loop does with a fixed-shape decode step.  The graph reads the pinned buffers at replay time.
@@ -332,7 +333,7 @@ def run_ours(args, rank, world, local_rank):
         side = torch.cuda.Stream()
         graphs = []
         with torch.cuda.stream(side):
-            for i in range(N_ROT):
+            for i in range(n_rot):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=side, capture_error_mode="thread_local"):
                     slim.slim_decode_step_host(runs[i].cache, q_h, k_h, v_h, out_h, staging, kv_len, B, max_kv, Hq,
@@ -341,13 +342,13 @@ def run_ours(args, rank, world, local_rank):
             out_h.zero_()
 
             def step_graph(i):
-                graphs[i % N_ROT].replay()
+                graphs[i % n_rot].replay()
                 side.synchronize()      # the caller needs the result before the next token
 
             for i in range(3):
                 step_graph(i)
             ok = torch.equal(out_h, out.cpu())
-            ms = statistics.median(timed_blocks(step_graph, args.steps, MIN_TIMED_MS / 2, side, barrier, world, dev))
+            ms = statistics.median(timed_blocks(step_graph, args.steps, args.min_ms / 2, side, barrier, world, dev))
         return ms, ok
 
     ms_e2e = ms_e2e_eager
@@ -386,7 +387,7 @@ def run_ours(args, rank, world, local_rank):
         "data": "synthetic",
         "config": {"workload": w.name, "batch_per_gpu": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128,
                    "context": ctx + 1, "cache": "int8 codes + fp32 scale per (token, kv head), 128-token pages",
-                   "l2": f"inputs larger than L2: {N_ROT} cache copies of {cache_bytes / 1e6:.0f} MB rotated",
+                   "l2": f"inputs larger than L2: {n_rot} cache copies of {cache_bytes / 1e6:.0f} MB rotated",
                    "parallelism": f"dp{world} (independent sequences per GPU, no collective)"},
         "hbm_gbs_step_per_gpu": step_bytes / (ms_total / args.steps * 1e-3) / 1e9,
         "pct_of_8tbs_step": 100.0 * step_bytes / (ms_total / args.steps * 1e-3) / 1e9 / 8000.0,
@@ -478,7 +479,7 @@ def run_sharded(args, rank, world, dev, barrier):
     if sampler:
         sampler.start()
         time.sleep(0.1)
-    blocks = timed_blocks(step, args.steps, MIN_TIMED_MS, stream, barrier, world, dev)
+    blocks = timed_blocks(step, args.steps, args.min_ms, stream, barrier, world, dev)
     clocks = sampler.stop() if sampler else None
     if rank != 0:
         return
@@ -729,6 +730,10 @@ def main():
                     help="divide ONE workload's decode attention over the ranks (strong scaling) instead of replicating workload 2")
     ap.add_argument("--shard-workload", type=int, default=4, choices=[2, 4, 5],
                     help="workload divided by --shard: 4 (by kv heads) or 5 (2 kv heads: by key ranges beyond 2 ranks)")
+    ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
+                    help="device time the repeated timed blocks must cover (default 200; small values for profiler runs)")
+    ap.add_argument("--copies", type=int, default=N_ROT,
+                    help="cache copies rotated between steps (default 12; fewer only for profiler captures that must stay small)")
     ap.add_argument("--extra-only", action="store_true",
                     help="run only the workload-3 prefill/append timings (for profiling that kernel) and print them")
     args = ap.parse_args()

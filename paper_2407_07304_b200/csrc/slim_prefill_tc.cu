@@ -446,9 +446,10 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     } else if (warp < 12 || warp >= 14) {
         // =========================================================== dequantise
         // A thread of warps 8-11 owns token row r = tid - 256 of every tile and converts its pieces 0..5 (a piece =
-        // 16 codes); a thread of warps 14, 15 owns rows 2 u, 2 u + 1 (u = tid - 448) and converts their pieces 6, 7.
+        // 16 codes); a thread of warps 14, 15 owns rows u and u + 64 (u = tid - 448) and converts their pieces 6, 7
+        // (consecutive lanes on consecutive rows: the swizzled 16-byte slots of a warp's access then cover all banks).
         const bool main_cv = warp < 12;
-        const int r0 = main_cv ? tid - 256 : 2 * (tid - 448);
+        const int r0 = main_cv ? tid - 256 : tid - 448;
         const int n_rows = main_cv ? 1 : 2, c_first = main_cv ? 0 : 6, c_last = main_cv ? 6 : 8;
         const bool announces = warp == 8 && lane == 0;   // the thread that publishes a tile's exponents
         for (int i = 0; i < 2 * NT; ++i) {
@@ -487,7 +488,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 if (q >= n_rows) break;
-                const int r = r0 + q;
+                const int r = r0 + 64 * q;
                 const float f = ((r < n_valid) ? scales[r] : 0.f) * rex;   // scale / 2^e in [0, 2)
                 const uint32_t fac2 = pack_half2(f, f);
                 unsigned char *dstb = dst_tile + r * 128;
