@@ -545,8 +545,17 @@ def extra_numbers(slim, workloads, dev):
             best = min(best, e0.elapsed_time(e1) / reps)
         return best
 
+    def both():
+        append()
+        prefill()
+
+    def step():
+        slim.slim_prefill_step(run.cache, q, k_new, v_new, out, cu, kvl, 1, S, S, w3.Hq, w3.sm_scale, run.ws_prefill, stream)
+
     ms_append = time_it(append, 20)
     ms_prefill = time_it(prefill, 5)
+    ms_both = time_it(both, 5)
+    ms_step = time_it(step, 5)
     flops = 4 * 128 * w3.Hq * S * (S + 1) // 2
     append_bytes = S * w3.Hkv * (2 * 256 + ROW_BYTES)
     hbm_peak, _, _ = _peaks()
@@ -717,6 +726,8 @@ def extra_numbers(slim, workloads, dev):
                        "frac_of_bf16_peak": flops / (ms_prefill * 1e-3) / 1e12 / bf16_peak,
                        "peak_tflops": bf16_peak, "peak_kind": f"of {peak_kind}",
                        "tokens_per_s_with_append": S / ((ms_prefill + ms_append) * 1e-3)},
+        # append + prefill of workload 3 as two calls back to back, and as the one call slim_prefill_step
+        "prefill_step_c3": {"workload": w3.name, "ms_two_calls": ms_both, "ms": ms_step, "tokens_per_s": S / (ms_step * 1e-3)},
         "append_c3": {"ms": ms_append, "gbs": append_bytes / (ms_append * 1e-3) / 1e9,
                       "frac_of_hbm_peak": append_bytes / (ms_append * 1e-3) / 1e9 / hbm_peak},
     }}

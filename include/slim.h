@@ -87,7 +87,7 @@ typedef struct slim_cache {
  * gets scale 0 and codes 0.  Codes and scale bits are reproducible exactly.
  *
  *   k_new, v_new  device bf16 [total_new][num_kv_heads][128], the new tokens of
- *                 all sequences concatenated in sequence order; 8-byte aligned
+ *                 all sequences concatenated in sequence order; 16-byte aligned
  *   cu_new        device int32 [B+1]: rows cu_new[b] .. cu_new[b+1]-1 belong to
  *                 sequence b (cu_new[0] == 0)
  *   start_pos     device int32 [B]: cache position of sequence b's first new token
@@ -130,6 +130,30 @@ int slim_kv_append(const slim_cache_t *cache, const void *k_new, const void *v_n
  *                  word (see slim_read_status) and should be zero
  */
 int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out,
+                      const int32_t *cu_q, const int32_t *kv_len,
+                      int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq, float sm_scale,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The first-token phase in one call (Section 2.2: K and V are written to the
+ * INT8 cache while the prompt is processed): exactly
+ *   slim_kv_append(cache, k_new, v_new, cu_q, start_pos, B, max_q, stream) with
+ *     start_pos[b] = kv_len[b] - (cu_q[b+1] - cu_q[b]), followed by
+ *   slim_attn_prefill(cache, q, out, cu_q, kv_len, ...),
+ * so kv_len[b] is the length of sequence b AFTER its new tokens, and every
+ * query row has a new K / V row at the same index.  Two kernels; the second
+ * is launched so that its set-up and its reads of q overlap the end of the
+ * first (programmatic dependent launch), and the codes it reads are still in
+ * the L2.  The rows are not quantised inside the attention kernel itself: a
+ * key tile is read by every row block behind it (up to 64 at 16384 tokens),
+ * each of which would have to quantise it again, or wait for the block that
+ * owns it, which the longest-first order of the row blocks rules out.
+ *
+ *   k_new, v_new  device bf16 [total_q][num_kv_heads][128], 16-byte aligned
+ *   other arguments, workspace and error behaviour as for slim_attn_prefill;
+ *   codes and scales written are bit for bit those of slim_kv_append.
+ */
+int slim_prefill_step(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new, void *out,
                       const int32_t *cu_q, const int32_t *kv_len,
                       int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq, float sm_scale,
                       void *workspace, size_t workspace_bytes, void *stream);

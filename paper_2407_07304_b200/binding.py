@@ -24,7 +24,7 @@ HEAD_DIM = 128
 PAGE_TOKENS = 128
 
 EXPORTS = (
-    "slim_kv_append", "slim_attn_prefill", "slim_attn_prefill_two_pass", "slim_attn_prefill_full_row", "slim_attn_decode", "slim_attn_decode_split",
+    "slim_kv_append", "slim_attn_prefill", "slim_prefill_step", "slim_attn_prefill_two_pass", "slim_attn_prefill_full_row", "slim_attn_decode", "slim_attn_decode_split",
     "slim_attn_decode_merge", "slim_attn_decode_static", "slim_static_status", "slim_static_reset",
     "slim_static_selftest_timeout", "slim_attn_decode_partial", "slim_attn_merge_partials", "slim_decode_step", "slim_decode_step_host", "slim_step_staging_bytes", "slim_read_status", "slim_selftest_timeout", "slim_workspace_bytes",
     "slim_cache_code_bytes", "slim_cache_scale_bytes", "slim_strerror", "slim_last_cuda_error",
@@ -73,6 +73,8 @@ def lib():
         L.slim_kv_append.restype = ctypes.c_int
         L.slim_attn_prefill.argtypes = [CP, P, P, P, P, I, I, I, I, F, P, Z, P]
         L.slim_attn_prefill.restype = ctypes.c_int
+        L.slim_prefill_step.argtypes = [CP, P, P, P, P, P, P, I, I, I, I, F, P, Z, P]
+        L.slim_prefill_step.restype = ctypes.c_int
         L.slim_attn_prefill_two_pass.argtypes = [CP, P, P, P, P, I, I, I, I, F, P, Z, P]
         L.slim_attn_prefill_two_pass.restype = ctypes.c_int
         L.slim_attn_prefill_full_row.argtypes = [CP, P, P, P, P, I, I, I, I, F, P, Z, P]
@@ -177,6 +179,13 @@ def slim_attn_prefill(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scal
     rc = lib().slim_attn_prefill(ctypes.byref(cache.struct), _ptr(q), _ptr(out), _ptr(cu_q), _ptr(kv_len),
                                  B, max_q, max_kv, Hq, sm_scale, _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "slim_attn_prefill")
+
+
+def slim_prefill_step(cache, q, k_new, v_new, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().slim_prefill_step(ctypes.byref(cache.struct), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(cu_q), _ptr(kv_len),
+                                 B, max_q, max_kv, Hq, sm_scale, _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "slim_prefill_step")
 
 
 def slim_attn_prefill_two_pass(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, sm_scale, workspace=None, stream=None):

@@ -15,7 +15,7 @@ int set_cuda_error(cudaError_t e)
 }
 
 int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
-                  const int32_t *start_pos, int B, int max_new, cudaStream_t stream);
+                  const int32_t *start_pos, int B, int max_new, cudaStream_t stream, const int32_t *len_after);
 int launch_decode_split(const slim_cache_t *c, const void *q, const void *k_new, const void *v_new, const int32_t *kv_len,
                         int B, int max_kv, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 int launch_decode_merge(const slim_cache_t *c, void *out, const int32_t *kv_len, int B, int max_kv, int Hq,
@@ -27,7 +27,7 @@ int launch_decode_partial(const slim_cache_t *c, const void *q, float *partial, 
 int launch_merge_partials(const float *parts, int R, int rows, void *out, cudaStream_t stream);
 size_t decode_workspace_bytes(int B, int Hq, int Hkv, int max_kv);
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
-                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass);
+                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass, bool after_append);
 int launch_prefill_row(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
                        int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream);
 size_t prefill_workspace_bytes();
@@ -55,9 +55,9 @@ SLIM_EXPORT int slim_kv_append(const slim_cache_t *cache, const void *k_new, con
     if (B < 0 || max_new < 0) return SLIM_ERR_INVALID_ARG;
     if (B == 0 || max_new == 0) return SLIM_OK;
     if (k_new == nullptr || v_new == nullptr || cu_new == nullptr || start_pos == nullptr) return SLIM_ERR_INVALID_ARG;
-    if (((uintptr_t)k_new & 7) || ((uintptr_t)v_new & 7)) return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15)) return SLIM_ERR_INVALID_ARG;   // rows are read 16 bytes at a time
     if (B > 65535) return SLIM_ERR_UNSUPPORTED;
-    return launch_append(cache, k_new, v_new, cu_new, start_pos, B, max_new, (cudaStream_t)stream);
+    return launch_append(cache, k_new, v_new, cu_new, start_pos, B, max_new, (cudaStream_t)stream, nullptr);
 }
 
 enum PrefillVariant { kPrefillStreamed, kPrefillTwoPass, kPrefillFullRow };
@@ -82,7 +82,31 @@ static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, co
         return launch_prefill_row(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream);
     }
     return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream,
-                             variant == kPrefillTwoPass);
+                             variant == kPrefillTwoPass, false);
+}
+
+// The first-token phase in one call: the prompt's K / V rows are quantised into the cache and the attention over
+// the cache follows, the second kernel launched so that its set-up and its query rows overlap the end of the first.
+SLIM_EXPORT int slim_prefill_step(const slim_cache_t *cache, const void *q, const void *k_new, const void *v_new, void *out,
+                                  const int32_t *cu_q, const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv,
+                                  int32_t Hq, float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    int rc = check_cache(cache);
+    if (rc != SLIM_OK) return rc;
+    if (B < 0 || max_q < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
+    if (Hq % cache->num_kv_heads != 0) return SLIM_ERR_UNSUPPORTED;
+    if (B == 0 || max_q == 0) return SLIM_OK;
+    if (q == nullptr || out == nullptr || cu_q == nullptr || kv_len == nullptr || k_new == nullptr || v_new == nullptr)
+        return SLIM_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15)) return SLIM_ERR_INVALID_ARG;
+    if (B > 65535 || Hq > 65535) return SLIM_ERR_UNSUPPORTED;
+    if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
+    const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
+    if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
+    // the new rows of sequence b go to positions kv_len[b] - q_len[b] ... kv_len[b] - 1
+    rc = launch_append(cache, k_new, v_new, cu_q, nullptr, B, max_q, (cudaStream_t)stream, kv_len);
+    if (rc != SLIM_OK) return rc;
+    return launch_prefill_tc(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream, false, true);
 }
 
 SLIM_EXPORT int slim_attn_prefill(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,

@@ -21,13 +21,15 @@ constexpr int kAppendRowsPerGroup = 1;     // rows in flight per group of lanes
 // NV = 16-byte loads per lane and row: 16 / NV lanes own a row.
 // grid = (ceil(max_new * Hkv / rows per block), B, 2 [K, V]); row index = token * Hkv + head within the
 // sequence's new rows.  step_tok / step_head = quotient and remainder of the block's group count by Hkv.
+// The first new token of sequence b goes to position start_pos[b], or, without start_pos, to len_after[b] minus the
+// sequence's new tokens (the caller states the lengths the sequences have after the append).
 template <int NV>
 __global__ void __launch_bounds__(kAppendThreads)
 slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
                    const int32_t *__restrict__ block_table,
                    const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
                    const int32_t *__restrict__ cu_new, const int32_t *__restrict__ start_pos,
-                   int Hkv, int max_pages_per_seq, int num_pages, int step_tok, int step_head)
+                   const int32_t *__restrict__ len_after, int Hkv, int max_pages_per_seq, int num_pages, int step_tok, int step_head)
 {
     constexpr int kLanes = 16 / NV;                       // lanes per row
     constexpr int kGroups = kAppendThreads / kLanes;      // rows the block handles per step
@@ -42,7 +44,7 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
     const int n_rows = (__ldg(cu_new + b + 1) - row0) * Hkv;
     const int first = (int)blockIdx.x * kRowsPerBlock;
     if (first >= n_rows) return;
-    const int start = __ldg(start_pos + b);
+    const int start = (start_pos != nullptr) ? __ldg(start_pos + b) : __ldg(len_after + b) - (__ldg(cu_new + b + 1) - row0);
     const uint4 *src = reinterpret_cast<const uint4 *>((kv ? v_new : k_new) + (size_t)row0 * Hkv * kHeadDim);
 
     // ---- every load first: the rows' data and the page ids of their destinations.  One division per thread:
@@ -86,7 +88,7 @@ slim_append_kernel(int8_t *__restrict__ codes, float *__restrict__ scales,
 }
 
 int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, const int32_t *cu_new,
-                  const int32_t *start_pos, int B, int max_new, cudaStream_t stream)
+                  const int32_t *start_pos, int B, int max_new, cudaStream_t stream, const int32_t *len_after)
 {
     constexpr int NV = kAppendNV;
     constexpr int kGroups = kAppendThreads / (16 / NV), kRowsPerBlock = kGroups * kAppendRowsPerGroup;
@@ -96,7 +98,7 @@ int launch_append(const slim_cache_t *c, const void *k_new, const void *v_new, c
     dim3 grid((unsigned)blocks, (unsigned)B, 2);
     slim_append_kernel<NV><<<grid, kAppendThreads, 0, stream>>>(
         c->codes, c->scales, c->block_table, static_cast<const __nv_bfloat16 *>(k_new),
-        static_cast<const __nv_bfloat16 *>(v_new), cu_new, start_pos, c->num_kv_heads, c->max_pages_per_seq,
+        static_cast<const __nv_bfloat16 *>(v_new), cu_new, start_pos, len_after, c->num_kv_heads, c->max_pages_per_seq,
         c->num_pages, kGroups / c->num_kv_heads, kGroups % c->num_kv_heads);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;

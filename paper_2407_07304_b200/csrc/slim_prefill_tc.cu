@@ -191,6 +191,9 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
     if (warp == 12 && lane == 0) {
         for (int i = 0; i < kPfRawStages; ++i) tc::mbar_init(bar(pfl::RAW_FULL, i), 1);
         tc::mbar_init_fence();
+        // everything above, and the other warps' set-up and query rows, may overlap the end of the kernel before
+        // this one in the stream (the append of the one-call prefill step); the cache is read from here on
+        pdl_wait();
         if (T > 0) {
             page_next = __ldg(p.block_table + (size_t)b * p.max_pages_per_seq);
             for (int i = 0; i < min(kPfRawStages, 2 * NT); ++i) request_raw(i);   // every stage is free the first time round
@@ -621,7 +624,7 @@ slim_prefill_tc_kernel(const __grid_constant__ CUtensorMap codes_map, const Pref
 size_t prefill_workspace_bytes() { return 16; }   // status word
 
 int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int32_t *cu_q, const int32_t *kv_len,
-                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass)
+                      int B, int max_q, int Hq, float sm_scale, void *workspace, cudaStream_t stream, bool two_pass, bool after_append)
 {
     PrefillTcParams p;
     p.scales = c->scales;
@@ -648,6 +651,7 @@ int launch_prefill_tc(const slim_cache_t *c, const void *q, void *out, const int
     if (p.n_qblocks > 65535 || B > 65535) return SLIM_ERR_UNSUPPORTED;
     dim3 grid((unsigned)Hq, (unsigned)B, (unsigned)p.n_qblocks);
     if (two_pass) slim_prefill_tc_kernel<true><<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
+    else if (after_append) SLIM_CUDA_TRY(launch_pdl(slim_prefill_tc_kernel<false>, grid, dim3(kPfThreads), pfl::kBytes, stream, map, p));
     else slim_prefill_tc_kernel<false><<<grid, kPfThreads, pfl::kBytes, stream>>>(map, p);
     SLIM_CUDA_TRY(cudaGetLastError());
     return SLIM_OK;

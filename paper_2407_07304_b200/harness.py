@@ -60,6 +60,23 @@ class LayerRun:
            self.ws_prefill)
         return [out[cu[b]:cu[b + 1]] for b in range(w.B)]
 
+    def prefill_step(self, counts, q_list):
+        """Append the next counts[b] rows of sequence b and attend q_list[b] (one query row per new token) over the
+        lengthened cache, in one library call."""
+        w = self.w
+        k_new = torch.cat([self.k[b][self.pos[b]:self.pos[b] + counts[b]] for b in range(w.B)]).contiguous()
+        v_new = torch.cat([self.v[b][self.pos[b]:self.pos[b] + counts[b]] for b in range(w.B)]).contiguous()
+        q = torch.cat([t.to(self.device) for t in q_list]).contiguous()
+        out = torch.empty_like(q)
+        cu = [0]
+        for c in counts:
+            cu.append(cu[-1] + c)
+        for b in range(w.B):
+            self.pos[b] += counts[b]
+        slim.slim_prefill_step(self.cache, q, k_new, v_new, out, self._i32(cu), self._i32(self.pos), w.B, max(counts),
+                               max(self.pos), w.Hq, w.sm_scale, self.ws_prefill)
+        return [out[cu[b]:cu[b + 1]] for b in range(w.B)]
+
     def decode(self, q):
         """One query token per sequence (bf16 [B, Hq, 128]) against the whole cache."""
         w = self.w

@@ -430,6 +430,60 @@ def test_chunked_prefill_offset_and_shuffled_pages():
         _assert_close(outs[b], want, f"chunked prefill seq {b}")
 
 
+def test_prefill_step_fresh_prompts_and_behind_a_cached_prefix():
+    # slim_prefill_step = slim_kv_append + slim_attn_prefill in one call: ragged prompts written and attended at once,
+    # then a second call whose new tokens sit behind the first call's (chunked prefill through a permuted block table)
+    from paper_2407_07304_b200 import binding as slim, harness
+    w = _custom(3, 8, 2, [333, 70, 258], [0, 0, 0], 0, 4242)
+    pages = w.pages_per_seq()
+    perm = torch.randperm(3 * pages + 2, generator=torch.Generator().manual_seed(5))[:3 * pages]
+    run = harness.LayerRun(w, block_table=perm.to(torch.int32).view(3, pages), num_pages=3 * pages + 2)
+    oc = _oracle_cache(w)
+    first = [200, 70, 129]
+    outs = run.prefill_step(first, [w.q_prefill[b][:first[b]] for b in range(3)])
+    torch.cuda.synchronize()
+    _assert_cache_bits(run, oc)
+    for b in range(3):
+        want = so.attention(bf16_bits(w.q_prefill[b][:first[b]]), *oc[b], first[b], w.sm_scale)
+        _assert_close(outs[b], want, f"prefill step, fresh prompt, seq {b}")
+    rest = [w.prefill_len[b] - first[b] for b in range(3)]   # 133, 0, 129: the second sequence adds nothing
+    outs = run.prefill_step(rest, [w.q_prefill[b][first[b]:] for b in range(3)])
+    torch.cuda.synchronize()
+    _assert_cache_bits(run, oc)
+    for b in range(3):
+        if rest[b] == 0:
+            continue
+        want = so.attention(bf16_bits(w.q_prefill[b][first[b]:]), *oc[b], w.prefill_len[b], w.sm_scale)
+        _assert_close(outs[b], want, f"prefill step behind a prefix, seq {b}")
+    assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
+
+
+def test_prefill_step_equals_append_then_prefill_bit_for_bit():
+    from paper_2407_07304_b200 import harness
+    w = workloads.make_workload(3, shrink=8)   # 1024 tokens, 32 heads
+    a, b_ = harness.LayerRun(w), harness.LayerRun(w)
+    a.append(w.prefill_len)
+    want = a.prefill(w.q_prefill)
+    got = b_.prefill_step(w.prefill_len, w.q_prefill)
+    torch.cuda.synchronize()
+    assert torch.equal(a.cache.codes, b_.cache.codes) and torch.equal(a.cache.scales, b_.cache.scales)
+    for x, y in zip(got, want):
+        assert torch.equal(x, y)
+
+
+def test_prefill_step_c1_all_outputs():
+    from paper_2407_07304_b200 import harness
+    w = workloads.make_workload(1)
+    run = harness.LayerRun(w)
+    oc = _oracle_cache(w)
+    outs = run.prefill_step(w.prefill_len, w.q_prefill)
+    torch.cuda.synchronize()
+    _assert_cache_bits(run, oc)
+    for b in range(w.B):
+        want = so.attention(bf16_bits(w.q_prefill[b]), *oc[b], w.prefill_len[b], w.sm_scale)
+        _assert_close(outs[b], want, f"prefill step workload 1 seq {b}")
+
+
 def test_empty_and_zero_length():
     from paper_2407_07304_b200 import binding as slim, harness
     w = _custom(2, 2, 1, [0, 0], [0, 5], 0, 500)
