@@ -287,16 +287,18 @@ int slim_decode_step(const slim_cache_t *cache, const void *q, const void *k_new
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * One decode step from host buffers: copies the step's query and new K/V rows
- * (one new token per sequence) host -> device, runs slim_decode_step and copies
+ * One decode step from host buffers: brings the step's query and new K/V rows
+ * (one new token per sequence) host -> device, runs slim_decode_step and brings
  * the result device -> host, all asynchronously on `stream` (Section 2.2: the
  * per-token step whose cache traffic Eq. 1 counts).  Host buffers should be pinned; they must stay
- * valid and out_host must not be read until the stream has been synchronised.
+ * valid and unchanged, and out_host must not be read, until the stream has been synchronised.
  *
- * If q_host, k_new_host and v_new_host lie back to back in one allocation (in that order) they are copied with
- * one transfer instead of three.  If out_host is pinned memory that the device can address (cudaHostAlloc,
- * cudaHostRegister) and 16-byte aligned, the kernel writes the result straight into it and no copy back is
- * issued; otherwise the result goes through `staging` and a device -> host copy.
+ * If the three input buffers are pinned memory that the device can address (cudaHostAlloc, cudaHostRegister)
+ * and 16-byte aligned, the kernel reads them where they are - every row crosses the bus once, as in a copy, but
+ * the step does not wait for a copy first.  Otherwise they are copied into `staging` (with one transfer instead
+ * of three if q_host, k_new_host and v_new_host lie back to back in one allocation, in that order).  If out_host
+ * is such pinned memory, the kernel writes the result straight into it and no copy back is issued; otherwise the
+ * result goes through `staging` and a device -> host copy.
  *
  * The call synchronises nothing and allocates nothing.  After one ordinary call with the same cache and shapes
  * (which creates the tensor map and sets the kernels' attributes) it may be recorded by stream capture into a

@@ -243,25 +243,33 @@ SLIM_EXPORT int slim_decode_step_host(const slim_cache_t *cache, const void *q_h
     char *d_q = static_cast<char *>(staging), *d_k = d_q + q_bytes, *d_v = d_k + kv_bytes, *d_o = d_v + kv_bytes;
     const char *hq = static_cast<const char *>(q_host), *hk = static_cast<const char *>(k_new_host),
                *hv = static_cast<const char *>(v_new_host);
-    if (hk == hq + q_bytes && hv == hk + kv_bytes) {
-        // the three host buffers are adjacent (one allocation): one copy instead of three
-        SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, hq, q_bytes + 2 * kv_bytes, cudaMemcpyHostToDevice, st));
-    } else {
-        SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, hq, q_bytes, cudaMemcpyHostToDevice, st));
-        SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, hk, kv_bytes, cudaMemcpyHostToDevice, st));
-        SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, hv, kv_bytes, cudaMemcpyHostToDevice, st));
-    }
-    // A pinned host buffer is mapped into the device's address space: the kernel then writes the result straight
-    // into it (visible to the host once the stream has been synchronised) and the copy back is not needed.
-    void *d_out = d_o;
-    cudaPointerAttributes attr;
-    if (cudaPointerGetAttributes(&attr, out_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
-        attr.devicePointer != nullptr && ((uintptr_t)attr.devicePointer & 15) == 0) {
-        d_out = attr.devicePointer;
-    } else {
+    // A pinned host buffer is mapped into the device's address space.  The kernel reads such inputs where they
+    // are (every row is read once, by one warp or one bulk copy: the step moves the same bytes over the bus as a
+    // copy would, without waiting for the copy first) and writes the result straight into such an output (visible
+    // to the host once the stream has been synchronised).  Ordinary host memory goes through the staging buffer.
+    auto mapped = [](const void *host) -> void * {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+            attr.devicePointer != nullptr && ((uintptr_t)attr.devicePointer & 15) == 0)
+            return attr.devicePointer;
         (void)cudaGetLastError();   // an unregistered host pointer is not an error here: it takes the copy
+        return nullptr;
+    };
+    const void *in_q = mapped(hq), *in_k = mapped(hk), *in_v = mapped(hv);
+    if (in_q == nullptr || in_k == nullptr || in_v == nullptr) {
+        if (hk == hq + q_bytes && hv == hk + kv_bytes) {
+            // the three host buffers are adjacent (one allocation): one copy instead of three
+            SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, hq, q_bytes + 2 * kv_bytes, cudaMemcpyHostToDevice, st));
+        } else {
+            SLIM_CUDA_TRY(cudaMemcpyAsync(d_q, hq, q_bytes, cudaMemcpyHostToDevice, st));
+            SLIM_CUDA_TRY(cudaMemcpyAsync(d_k, hk, kv_bytes, cudaMemcpyHostToDevice, st));
+            SLIM_CUDA_TRY(cudaMemcpyAsync(d_v, hv, kv_bytes, cudaMemcpyHostToDevice, st));
+        }
+        in_q = d_q, in_k = d_k, in_v = d_v;
     }
-    rc = launch_decode(cache, d_q, d_k, d_v, d_out, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
+    void *d_out = mapped(out_host);
+    if (d_out == nullptr) d_out = d_o;
+    rc = launch_decode(cache, in_q, in_k, in_v, d_out, kv_len, B, max_kv, Hq, sm_scale, workspace, st);
     if (rc != SLIM_OK) return rc;
     if (d_out == d_o) SLIM_CUDA_TRY(cudaMemcpyAsync(out_host, d_o, q_bytes, cudaMemcpyDeviceToHost, st));
     return SLIM_OK;

@@ -519,6 +519,19 @@ def test_bad_arguments_are_rejected_on_the_host():
     with pytest.raises(slim.SlimError) as e:
         slim.slim_attn_decode(run.cache, q, q.clone(), kvl, 1, 100000, 4, 1.0, run.ws_decode)  # beyond the page table
     assert e.value.code == slim.SLIM_ERR_INVALID_ARG
+    # rows are read 16 bytes at a time: inputs that are only 8-byte aligned are refused, not read
+    kn = torch.zeros((1 * 2 * 128 + 4,), dtype=torch.bfloat16, device="cuda")
+    cu = torch.tensor([0, 1], dtype=torch.int32, device="cuda")
+    pos = torch.tensor([10], dtype=torch.int32, device="cuda")
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_kv_append(run.cache, kn[4:], kn[:256], cu, pos, 1, 1)
+    assert e.value.code == slim.SLIM_ERR_INVALID_ARG
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_prefill_step(run.cache, q, None, kn[:256], q.clone(), cu, kvl, 1, 1, 10, 4, 1.0, run.ws_prefill)
+    assert e.value.code == slim.SLIM_ERR_INVALID_ARG
+    with pytest.raises(slim.SlimError) as e:
+        slim.slim_prefill_step(run.cache, q, kn[4:], kn[:256], q.clone(), cu, kvl, 1, 1, 10, 4, 1.0, run.ws_prefill)
+    assert e.value.code == slim.SLIM_ERR_INVALID_ARG
     torch.cuda.synchronize()
 
 
@@ -592,10 +605,11 @@ def test_status_words_stay_clear():
     assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
 
 
-@pytest.mark.parametrize("pinned_out", [True, False])
-def test_decode_step_from_host_buffers(pinned_out):
-    # slim_decode_step_host: H2D copy, the one-kernel step, and the result either written by the kernel into the
-    # pinned host buffer or, for ordinary host memory, copied back through the staging buffer
+@pytest.mark.parametrize("pinned_in,pinned_out", [(True, True), (True, False), (False, True), (False, False)])
+def test_decode_step_from_host_buffers(pinned_in, pinned_out):
+    # slim_decode_step_host: pinned inputs are read by the kernel where they are, ordinary host memory is copied into
+    # the staging buffer first; the result is either written by the kernel into the pinned host buffer or, for
+    # ordinary host memory, copied back through the staging buffer
     from paper_2407_07304_b200 import binding as slim, harness
     w = workloads.make_workload(4, shrink=16)
     run = harness.LayerRun(w)
@@ -603,9 +617,10 @@ def test_decode_step_from_host_buffers(pinned_out):
     dev = run.device
     B, Hq, Hkv = w.B, w.Hq, w.Hkv
     ctx = list(run.pos)
-    k_new = torch.stack([w.k[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
-    v_new = torch.stack([w.v[b][ctx[b]] for b in range(B)]).contiguous().pin_memory()
-    q = w.q_decode[0].contiguous().pin_memory()
+    pin = (lambda t: t.pin_memory()) if pinned_in else (lambda t: t.clone())
+    k_new = pin(torch.stack([w.k[b][ctx[b]] for b in range(B)]).contiguous())
+    v_new = pin(torch.stack([w.v[b][ctx[b]] for b in range(B)]).contiguous())
+    q = pin(w.q_decode[0].contiguous())
     out = torch.zeros_like(q).pin_memory() if pinned_out else torch.zeros(q.shape, dtype=q.dtype)
     staging = torch.empty(slim.slim_step_staging_bytes(B, Hq, Hkv), dtype=torch.uint8, device=dev)
     kv_len = torch.tensor(ctx, dtype=torch.int32, device=dev) + 1
