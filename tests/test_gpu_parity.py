@@ -320,8 +320,10 @@ def test_ragged_lengths_prefill_and_decode(lens):
     _check(_custom(B, 4, 2, lens, [0] * B, 2, 100 + lens[0]))
 
 
-@pytest.mark.parametrize("Hq,Hkv", [(1, 1), (8, 1), (16, 1), (12, 3), (6, 2)])
+@pytest.mark.parametrize("Hq,Hkv", [(1, 1), (8, 1), (16, 1), (12, 3), (6, 2), (4, 2), (10, 2), (7, 1), (9, 1), (13, 1), (30, 2)])
 def test_group_sizes(Hq, Hkv):
+    # 1, 2, 3, 4, 5, 7, 8 query heads per kv head (the eight-head kernel, some of its operand rows empty) and
+    # 9, 13, 15, 16 (the sixteen-head kernel)
     _check(_custom(2, Hq, Hkv, [70, 200], [37, 0], 2, 200 + Hq))
 
 
@@ -595,6 +597,14 @@ def test_one_call_step_many_short_sequences():
     B = 300
     lens = [(7 * i) % 40 + 1 for i in range(B)]
     _check(_custom(B, 4, 2, [0] * B, [n - 1 for n in lens], 2, 950), one_call_step=True)
+
+
+def test_more_pairs_than_the_split_kernel_counts():
+    # 2100 sequences x 8 kv heads = 16800 (sequence, kv head) pairs: more than the 16384 counters of the split kernel's
+    # own merge, so the merge kernel follows; lengths 1..40, two one-call steps
+    B = 2100
+    lens = [(11 * i) % 40 + 1 for i in range(B)]
+    _check(_custom(B, 8, 8, [0] * B, [n - 1 for n in lens], 2, 951), one_call_step=True)
 
 
 def test_status_words_stay_clear():
