@@ -62,10 +62,12 @@ SLIM_EXPORT int slim_kv_append(const slim_cache_t *cache, const void *k_new, con
 
 enum PrefillVariant { kPrefillStreamed, kPrefillTwoPass, kPrefillFullRow };
 
-static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
-                         const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
-                         float sm_scale, void *workspace, size_t workspace_bytes, void *stream, PrefillVariant variant)
+// Shared validation of the prefill entry points; *launch is false for a valid no-op.
+static int check_prefill(const slim_cache_t *cache, const void *q, const void *out, const int32_t *cu_q, const int32_t *kv_len,
+                         int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq, const void *workspace, size_t workspace_bytes,
+                         bool *launch)
 {
+    *launch = false;
     int rc = check_cache(cache);
     if (rc != SLIM_OK) return rc;
     if (B < 0 || max_q < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
@@ -77,6 +79,17 @@ static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, co
     if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
     const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
     if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
+    *launch = true;
+    return SLIM_OK;
+}
+
+static int prefill_entry(const slim_cache_t *cache, const void *q, void *out, const int32_t *cu_q,
+                         const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv, int32_t Hq,
+                         float sm_scale, void *workspace, size_t workspace_bytes, void *stream, PrefillVariant variant)
+{
+    bool launch;
+    const int rc = check_prefill(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
     if (variant == kPrefillFullRow) {
         if (max_kv > SLIM_FULL_ROW_MAX_KEYS) return SLIM_ERR_UNSUPPORTED;   // the score strip of a row block must fit tensor memory
         return launch_prefill_row(cache, q, out, cu_q, kv_len, B, max_q, Hq, sm_scale, workspace, (cudaStream_t)stream);
@@ -91,18 +104,10 @@ SLIM_EXPORT int slim_prefill_step(const slim_cache_t *cache, const void *q, cons
                                   const int32_t *cu_q, const int32_t *kv_len, int32_t B, int32_t max_q, int32_t max_kv,
                                   int32_t Hq, float sm_scale, void *workspace, size_t workspace_bytes, void *stream)
 {
-    int rc = check_cache(cache);
-    if (rc != SLIM_OK) return rc;
-    if (B < 0 || max_q < 0 || max_kv < 0 || Hq <= 0) return SLIM_ERR_INVALID_ARG;
-    if (Hq % cache->num_kv_heads != 0) return SLIM_ERR_UNSUPPORTED;
-    if (B == 0 || max_q == 0) return SLIM_OK;
-    if (q == nullptr || out == nullptr || cu_q == nullptr || kv_len == nullptr || k_new == nullptr || v_new == nullptr)
-        return SLIM_ERR_INVALID_ARG;
-    if (((uintptr_t)q & 15) || ((uintptr_t)out & 15) || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15)) return SLIM_ERR_INVALID_ARG;
-    if (B > 65535 || Hq > 65535) return SLIM_ERR_UNSUPPORTED;
-    if ((long long)max_kv > (long long)cache->max_pages_per_seq * SLIM_PAGE_TOKENS) return SLIM_ERR_INVALID_ARG;
-    const size_t need = slim_workspace_bytes(SLIM_PHASE_PREFILL, B, Hq, cache->num_kv_heads, max_q, max_kv);
-    if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SLIM_ERR_WORKSPACE;
+    bool launch;
+    int rc = check_prefill(cache, q, out, cu_q, kv_len, B, max_q, max_kv, Hq, workspace, workspace_bytes, &launch);
+    if (rc != SLIM_OK || !launch) return rc;
+    if (k_new == nullptr || v_new == nullptr || ((uintptr_t)k_new & 15) || ((uintptr_t)v_new & 15)) return SLIM_ERR_INVALID_ARG;
     // the new rows of sequence b go to positions kv_len[b] - q_len[b] ... kv_len[b] - 1
     rc = launch_append(cache, k_new, v_new, cu_q, nullptr, B, max_q, (cudaStream_t)stream, kv_len);
     if (rc != SLIM_OK) return rc;

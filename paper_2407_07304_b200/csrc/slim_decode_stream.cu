@@ -6,9 +6,11 @@
 //
 //  * One thread block per SM.  The work - every 256-token chunk of every (sequence, kv head) - is cut
 //    into one contiguous range per block.  A chunk is the unit of a partial result (m, l, O[128]).
-//  * One warp is the producer: one thread walks the block's chunks and asks the TMA engine for each
-//    chunk's INT8 K tiles and V tiles into a ring of 16 KB tile stages (128-byte swizzled, completion
-//    counted on mbarriers) and for its scales and query rows into a small ring of chunk records.  A
+//  * Two producer threads, each in a warp of its own, walk the block's chunks: one asks the TMA engine
+//    for each chunk's INT8 K tiles and V tiles into a ring of 16 KB tile stages (128-byte swizzled,
+//    completion counted on mbarriers), the other for its scales and query rows into a small ring of
+//    chunk records (one thread hands the copy engine about one request per 100 ns, which alone would
+//    limit the stream).  Their two warps also find the block's range, one its start and one its end.  A
 //    stage goes back to the producer the moment the tensor cores have read it (the MMA completion
 //    itself arrives on the stage's mbarrier), so K tiles are held only until the scores are out and
 //    most of the ring is in flight at any time.  A ragged last tile is fetched in 16-row boxes so
