@@ -460,6 +460,41 @@ def test_prefill_step_fresh_prompts_and_behind_a_cached_prefix():
     assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
 
 
+def test_prefill_step_random_prompts_in_two_parts_through_permuted_pages():
+    # forty seeded random batches: every prompt is written and attended in two calls (either part may be empty, so a call
+    # mixes fresh prompts, continued ones and sequences without new tokens), pages in a random order
+    import random
+    from paper_2407_07304_b200 import binding as slim, harness
+    rng = random.Random(2407)
+    for it in range(40):
+        B = rng.choice([1, 2, 3, 4, 7])
+        Hkv = rng.choice([1, 2, 4, 8])
+        G = rng.choice([1, 2, 4, 8, 16])
+        lens = [rng.choice([1, 2, 127, 128, 129, 255, 256, 257, 300, 511, 513, rng.randint(1, 1500)]) for _ in range(B)]
+        w = _custom(B, Hkv * G, Hkv, lens, [0] * B, 0, rng.randint(0, 10 ** 6))
+        pages = w.pages_per_seq()
+        extra = rng.randint(0, 5)
+        perm = torch.randperm(B * pages + extra, generator=torch.Generator().manual_seed(rng.randint(0, 10 ** 6)))[:B * pages]
+        run = harness.LayerRun(w, block_table=perm.to(torch.int32).view(B, pages), num_pages=B * pages + extra)
+        oc = _oracle_cache(w)
+        first = [rng.choice([0, n, rng.randint(0, n)]) for n in lens]
+        if sum(first) == 0:
+            first[0] = lens[0]
+        done = [0] * B
+        for part in (first, [lens[b] - first[b] for b in range(B)]):
+            if sum(part) == 0:
+                continue
+            outs = run.prefill_step(part, [w.q_prefill[b][done[b]:done[b] + part[b]] for b in range(B)])
+            torch.cuda.synchronize()
+            for b in range(B):
+                if part[b] > 0:
+                    want = so.attention(bf16_bits(w.q_prefill[b][done[b]:done[b] + part[b]]), *oc[b], done[b] + part[b], w.sm_scale)
+                    _assert_close(outs[b], want, f"problem {it} seq {b}")
+                    done[b] += part[b]
+        _assert_cache_bits(run, oc)
+        assert slim.slim_read_status(run.ws_prefill) == slim.SLIM_OK
+
+
 def test_prefill_step_equals_append_then_prefill_bit_for_bit():
     from paper_2407_07304_b200 import harness
     w = workloads.make_workload(3, shrink=8)   # 1024 tokens, 32 heads
