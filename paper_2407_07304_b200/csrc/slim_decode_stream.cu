@@ -611,9 +611,9 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 uint32_t ph[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int gi = tile0 + i;
-                    st[i] = gi % S;
-                    ph[i] = (uint32_t)(gi / S) & 1u;
+                    const unsigned gi = (unsigned)(tile0 + i);   // (unsigned: after a wait that ran out the record may hold anything, and the stage index must stay inside the ring)
+                    st[i] = (int)(gi % (unsigned)S);
+                    ph[i] = (gi / (unsigned)S) & 1u;
                 }
                 // ---- scores: S^T[token][head] = K_codes . Q^T; each K stage goes back to the producer when read
 #pragma unroll
@@ -709,6 +709,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
             wait(bar_info_full(islot), iph);
             const int *meta = reinterpret_cast<const int *>(info + L::kMeta);
             const int b = meta[0], head = meta[1], chunk = meta[2], n_tok = meta[3];
+            const bool record_ok = ok;   // false: the wait for the record ran out and its fields may hold anything - nothing is written to global memory from them
             const int n_tiles = n_tok > kStTile ? 2 : 1;
             const int h0 = head * p.G;
 
@@ -847,7 +848,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int h = 0; h < NH; ++h) {
-                    if (h < p.G) {
+                    if (h < p.G && record_ok) {
                         const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_slots + chunk;
                         p.part_o[ps * kHeadDim + gtid] = (float)(((int)r[h] << 8) + (int)r[NH + h]) * (1.f / kStPFix);
                     }
@@ -867,7 +868,7 @@ slim_decode_stream_kernel(const __grid_constant__ CUtensorMap map_tile, const __
                 }
 #pragma unroll
                 for (int o = kLanesPerHead / 2; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-                if (seg == 0 && h < p.G) {
+                if (seg == 0 && h < p.G && record_ok) {
                     const size_t ps = ((size_t)b * p.Hq + h0 + h) * p.n_slots + chunk;
                     const float4 mw = *reinterpret_cast<const float4 *>(red_m + h * 4);
                     p.part_ml[ps * 2] = fmaxf(fmaxf(mw.x, mw.y), fmaxf(mw.z, mw.w));
